@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Throughput of batched schedule evaluation: schedule-steps evaluated per second.
+
+One "step" of the benchmark is one pass of the whole evaluation (offsets, occurrence table, free
+steps, memory profile, reductions) over one batch of B candidate sequences, through the C ABI.
+Workload: the training-graph-shaped configuration n=442, m=1247, B=16384, C=2, budget = 80 % of the
+no-rematerialization peak.  Inputs are synthetic and seeded; a ring of distinct batches larger than
+the L2 cache is cycled so that every timed pass reads its sequences from HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (under torchrun) every rank evaluates its own ring of batches on its own GPU: sequences
+are independent, no collective is on the data path; the reported value is the total over ranks
+divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD_IDX = 2
+METRIC = "schedule_steps_per_s_n442_B16384"
+UNIT = "steps/s"
+PCT = 80
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def make_ring(workloads, n_batches, rank):
+    """Distinct batches of the benchmark configuration (same graph, different schedule seeds)."""
+    base = workloads.make(WORKLOAD_IDX, seed=1)
+    s = workloads.spec(WORKLOAD_IDX)
+    ring = [(base.seqs, base.lens)]
+    for k in range(1, n_batches):
+        seqs, lens = workloads.schedules(base.n, base.edges, base.C, s["p"], s["B"],
+                                         seed=100003 * (rank + 1) + k, t_cap=base.meta["t_cap"])
+        ring.append((seqs, lens))
+    return base, ring
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2304_14463_b200 import workloads
+    from oracle import OracleGraph
+    base = workloads.make(WORKLOAD_IDX, seed=1)
+    O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
+    cores = len(os.sched_getaffinity(0))
+    P0 = O.eval(np.arange(base.n), 1 << 62)["peak"]
+    M = P0 * PCT // 100
+    for _ in range(args.warmup):
+        O.eval_batch(base.seqs, base.lens, M, n_threads=cores)
+    t0 = time.perf_counter()
+    used = cores
+    for _ in range(args.steps):
+        _, _, _, used = O.eval_batch(base.seqs, base.lens, M, n_threads=cores)
+    dt = time.perf_counter() - t0
+    steps = base.total_steps * args.steps
+    value = steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic",
+            "config": {"workload": f"{base.name}: n={base.n} m={len(base.edges)} B={base.B} C={base.C} "
+                                   f"M={PCT}% of no-remat peak", "sum_T": base.total_steps},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle",
+                             "sample": f"the full batch ({base.B} sequences, {base.total_steps} steps) per step, "
+                                       f"{args.steps} steps"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def time_oracle(base, M, budget_s=6.0):
+    from oracle import OracleGraph
+    O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
+    cores = len(os.sched_getaffinity(0))
+    O.eval_batch(base.seqs, base.lens, M, n_threads=cores)
+    out = {}
+    for label, threads, share in (("all", cores, 0.6), ("one", 1, 0.4)):
+        reps, t0 = 0, time.perf_counter()
+        used = threads
+        while True:
+            res = O.eval_batch(base.seqs, base.lens, M, n_threads=threads)
+            used = res[3]
+            reps += 1
+            dt = time.perf_counter() - t0
+            if dt > budget_s * share and reps >= 2:
+                break
+        out[label] = (base.total_steps * reps / dt, used, reps, res)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ring", type=int, default=16, help="distinct input batches cycled through")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 5 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args)
+    args.steps = 4000 if args.steps is None else args.steps
+    args.warmup = max(3, 200 if args.warmup is None else args.warmup)
+
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    import __graft_entry__
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2304_14463_b200 import binding, workloads
+
+    base, ring_host = make_ring(workloads, args.ring, rank)
+    G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
+    M = binding.budget_from_peak(G.no_remat_peak(), PCT)
+    ring = []
+    for seqs, lens in ring_host:
+        B = len(lens)
+        ring.append(dict(seqs=torch.from_numpy(seqs).cuda(), lens=torch.from_numpy(lens).cuda(),
+                         peak=torch.empty(B, dtype=torch.int64, device="cuda"),
+                         dur=torch.empty(B, dtype=torch.int64, device="cuda"),
+                         st=torch.empty(B, dtype=torch.int32, device="cuda"),
+                         steps=int(lens.sum()), B=B))
+    ring_bytes = sum(4 * r["steps"] + 4 * r["B"] for r in ring)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        r = ring[i % len(ring)]
+        G.eval_batch(r["seqs"], r["lens"], M, out_peak=r["peak"], out_dur=r["dur"], out_feasible=r["st"])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput: K steps back to back on one stream
+    for i in range(args.warmup):
+        step(i)
+    launches_per_step = binding.moc_last_launch_count()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+    ms = e0.elapsed_time(e1)
+    steps_done = sum(ring[i % len(ring)]["steps"] for i in range(args.steps))
+
+    # ---- the same region again with an event pair around every call, to get the per-launch time
+    # of the evaluation kernel (the offsets kernel is timed separately and subtracted)
+    n_k = min(args.steps, 512)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
+    for i in range(n_k):
+        evs[i][0].record(stream)
+        step(i)
+        evs[i][1].record(stream)
+    torch.cuda.synchronize()
+    call_ms = np.array([a.elapsed_time(b) for a, b in evs])
+
+    # ---- end to end: host buffers in, host buffers out, through the host entry point
+    hr = []
+    for seqs, lens in ring_host[:4]:
+        B = len(lens)
+        hr.append(dict(seqs=torch.from_numpy(seqs).pin_memory(), lens=torch.from_numpy(lens).pin_memory(),
+                       peak=torch.empty(B, dtype=torch.int64).pin_memory(),
+                       dur=torch.empty(B, dtype=torch.int64).pin_memory(),
+                       st=torch.empty(B, dtype=torch.int32).pin_memory(), steps=int(lens.sum()), B=B))
+    n_e2e = max(3, min(args.steps, 64))
+    for i in range(3):
+        r = hr[i % len(hr)]
+        G.eval_batch_host(r["seqs"], r["lens"], M, r["peak"], r["dur"], r["st"])
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps = 0
+    for i in range(n_e2e):
+        r = hr[i % len(hr)]
+        G.eval_batch_host(r["seqs"], r["lens"], M, r["peak"], r["dur"], r["st"])
+        e2e_steps += r["steps"]
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+        tot = torch.tensor([steps_done, e2e_steps], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+        steps_done, e2e_steps = float(tot[0]), float(tot[1])
+
+    if rank == 0:
+        peak_gbs, peak_kind = load_peaks()
+        r0 = ring[0]
+        alg_bytes = 4 * r0["steps"] + 4 * r0["B"] + 20 * r0["B"]
+        kernel_ms = float(np.median(call_ms))
+        info = G.info()
+        line = {
+            "metric": METRIC, "value": steps_done / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64" if info["wide"] else "int32", "data": "synthetic",
+            "config": {"workload": f"{base.name}: n={base.n} m={len(base.edges)} B={base.B} C={base.C} "
+                                   f"M={PCT}% of no-remat peak ({M})",
+                       "sum_T_per_step": r0["steps"], "cold_l2": f"ring of {len(ring)} distinct batches, "
+                       f"{ring_bytes / 1e6:.0f} MB of inputs > {L2_BYTES / 1e6:.0f} MB L2",
+                       "per_gpu_batch": base.B},
+            "gpu_launches": launches_per_step * args.steps,
+            "e2e": {"value": e2e_steps / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": 4 * hr[0]["steps"] + 4 * hr[0]["B"], "d2h_bytes_per_step": 20 * hr[0]["B"],
+                    "steps": n_e2e, "api": "moc_eval_batch_host (pinned host buffers)"},
+            "roofline": {"bound": "hbm", "achieved": alg_bytes / (kernel_ms * 1e-3) / 1e9, "peak": peak_gbs,
+                         "unit": "GB/s", "frac": alg_bytes / (kernel_ms * 1e-3) / 1e9 / peak_gbs,
+                         "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": kernel_ms,
+                         "kernel": "eval kernel + offsets kernel of one call (event pair around the call)"},
+            "clocks": clocks.summary(),
+        }
+        if not args.no_cpu_baseline:
+            o = time_oracle(base, M)
+            res = o["all"][3]
+            torch.cuda.synchronize()
+            same = bool((ring[0]["peak"].cpu().numpy() == res[0]).all() and (ring[0]["dur"].cpu().numpy() == res[1]).all()
+                        and (ring[0]["st"].cpu().numpy() == res[2]).all())
+            line["cpu_baseline"] = {"value": o["all"][0], "unit": UNIT, "cores": o["all"][1], "kind": "oracle",
+                                    "sample": f"the full first batch ({base.B} sequences, {base.total_steps} steps), "
+                                              f"{o['all'][2]} passes on all cores",
+                                    "one_core_value": o["one"][0]}
+            line["parity_first_batch"] = same
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,148 @@
+/*
+ * moc -- batched evaluation of rematerialization sequences on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the shared library libmoc_b200.so.  The operations are those of the rematerialization
+ * problem of "Moccasin: Efficient Tensor Rematerialization for Neural Networks" (arXiv 2304.14463):
+ * given a compute DAG G=(V,E) with per-node duration w_v and output size m_v, and a candidate
+ * execution sequence in which every node runs between 1 and C times, report the total duration,
+ * the peak memory footprint and whether the sequence meets the data dependencies and a memory
+ * budget M (Section 1, problem statement; Section 2, Eqs. 1-8).
+ *
+ * Conventions
+ *   - nodes are 0..n-1; an edge (u,v) means "v consumes the output of u" (Section 1);
+ *   - a sequence seq[0..T) lists node ids in execution order; position t is the t-th *filled*
+ *     compute event of Section 2 (empty events contribute to neither duration nor peak);
+ *   - each occurrence ("copy") of a node is one active retention interval [s,e] of Section 2 with
+ *     s = its position; its end e ("free step") is the last step that consumes this copy before
+ *     the node is computed again (Eq. 3: intervals of one node do not overlap; Eq. 5: a consumer
+ *     at step t needs a copy with s+1 <= t <= e, and the most recent earlier copy is the one
+ *     charged, which makes every interval as short as the sequence permits); a copy nobody
+ *     consumes has e = s (Eq. 2); the last copy of a node without successors is the result of the
+ *     computation and stays resident to step T-1;
+ *   - memory in use at step t is the sum of m over the copies with s <= t <= e, both ends
+ *     inclusive (Eq. 4); the peak is the maximum over the steps (Section 2).
+ *
+ * Per-sequence status codes (never an error return; bad sequences cannot fault the GPU):
+ *     1  dependencies met and peak <= M                      peak, duration valid
+ *     0  dependencies met, peak > M                           peak, duration valid
+ *    -1  some consumer has no earlier copy of a predecessor  peak = -1, duration valid (Eq. 5)
+ *    -2  malformed: length outside [n, C*n], id outside [0,n), a node absent (Eq. 7) or computed
+ *        more than C times (Section 2, C_v)                  peak = duration = -1
+ *
+ * Every function returns MOC_OK or a negative error code and never throws or aborts;
+ * moc_last_error() gives the text for the calling thread.  "HOST" / "DEVICE" below says where a
+ * pointer must live.  The caller owns every array; the library owns the handle, its device copy
+ * of the graph and grow-only scratch attached to the handle.  Because of that scratch, calls on
+ * one handle must be ordered (issue them from one thread, on one stream, or synchronise between
+ * streams); different handles are independent.  There is no CPU fallback: without a CUDA device
+ * every call that needs one fails with MOC_ERR_CUDA.
+ */
+#ifndef MOC_H_
+#define MOC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOC_OK 0
+#define MOC_ERR_ARG (-1)      /* null pointer, negative size, value outside its documented range   */
+#define MOC_ERR_RANGE (-2)    /* edge endpoint outside [0,n)                                       */
+#define MOC_ERR_CYCLE (-3)    /* self-loop or directed cycle                                       */
+#define MOC_ERR_OVERFLOW (-4) /* negative weight, or 8*sum(w) or 8*sum(m) would not fit in 62 bits  */
+#define MOC_ERR_CUDA (-5)     /* a CUDA runtime call failed (text in moc_last_error)               */
+#define MOC_ERR_NOMEM (-6)    /* host or device allocation failed                                  */
+
+#define MOC_MAX_COPIES 8      /* largest admissible C                                              */
+
+typedef struct moc_graph moc_graph; /* opaque */
+
+/*
+ * Problem data of Section 1: DAG, durations, output sizes.
+ *   n        number of nodes, >= 1
+ *   n_edges  number of (u,v) pairs in `edges`, >= 0
+ *   edges    HOST, 2*n_edges ints, pair k = (edges[2k], edges[2k+1]) = (u,v): v consumes u.
+ *            Duplicates are accepted and merged.  May be NULL when n_edges == 0.
+ *   w, m     HOST, n values each, all >= 0 (opaque integer units).
+ *   out      receives the handle; device copies live on the CUDA device current at the call.
+ * Errors: MOC_ERR_ARG, MOC_ERR_RANGE, MOC_ERR_CYCLE, MOC_ERR_OVERFLOW, MOC_ERR_CUDA,
+ * MOC_ERR_NOMEM; *out is NULL on error.  Synchronous (copies the graph before returning).
+ * The maximum number of copies per node starts at C = 2 (Section 4.3 uses C_v = 2 throughout).
+ */
+int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int64_t* w,
+                     const int64_t* m, moc_graph** out);
+
+/* Sets the cap C on copies per node (the paper's C_v, uniform over nodes; Section 2).
+ * 1 <= C <= MOC_MAX_COPIES, else MOC_ERR_ARG. */
+int moc_graph_set_max_copies(moc_graph* g, int32_t C);
+
+/* Frees the handle with its device memory.  NULL is accepted.  The caller must have
+ * synchronised every stream that still runs work of this handle. */
+void moc_graph_destroy(moc_graph* g);
+
+/* Facts about a handle (any pointer may be NULL): node count, number of distinct edges, current
+ * C, and whether memory sums are accumulated in 64 bits (1) or provably fit 32 bits (0) at that C. */
+int moc_graph_info(const moc_graph* g, int32_t* n, int64_t* n_edges, int32_t* C, int32_t* wide);
+
+/*
+ * Evaluates B sequences (objective Eq. 1, memory constraint Eq. 4, precedence Eq. 5, peak as
+ * defined in Section 2).
+ *   seqs          DEVICE, int32, packed back to back: sequence b occupies
+ *                 seqs[offs[b] .. offs[b]+len_b) with len_b = max(lens[b], 0) and offs the
+ *                 exclusive prefix sum of len_b.  Must hold sum(len_b) ints, 4-byte aligned.
+ *   lens          DEVICE, B ints.
+ *   B             number of sequences, >= 0 (0: nothing is launched, MOC_OK).
+ *   M             memory budget.
+ *   out_peak      DEVICE, B int64: peak memory footprint (or -1, see status codes).
+ *   out_dur       DEVICE, B int64: total duration with recomputations (or -1).
+ *   out_feasible  DEVICE, B int32: status code 1 / 0 / -1 / -2.
+ *   stream        a cudaStream_t (NULL = default stream).  The call only enqueues work; outputs
+ *                 are valid once the stream has been synchronised.
+ * Errors: MOC_ERR_ARG (null pointer with B > 0, B < 0), MOC_ERR_CUDA, MOC_ERR_NOMEM (scratch
+ * growth; happens only when B exceeds every earlier B on this handle).
+ */
+int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B,
+                   int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
+                   void* stream);
+
+/*
+ * Same evaluation with every array in HOST memory (pinned memory makes the copies asynchronous
+ * with respect to the host, pageable memory works too): copies seqs (n_steps ints, which must be
+ * at least sum(max(lens[b],0))) and lens to device staging owned by the handle, evaluates, copies
+ * the three outputs back and synchronises `stream` before returning.
+ */
+int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps,
+                        const int32_t* lens, int32_t B, int64_t M, int64_t* out_peak,
+                        int64_t* out_dur, int32_t* out_feasible, void* stream);
+
+/*
+ * Memory profile of one sequence (the per-event sums of Eq. 4 and the interval ends of Section 2).
+ *   seq          DEVICE, len int32 node ids.
+ *   out_profile  DEVICE, len int64: memory in use at every step.
+ *   out_free     DEVICE, len int32: free step of the copy executed at each step; may be NULL.
+ *   out_status   DEVICE, 1 int32: -2 / -1 as above, otherwise 1.  When the status is negative
+ *                both arrays are filled with -1.
+ * Asynchronous on `stream` like moc_eval_batch.  len < 0 is MOC_ERR_ARG.
+ */
+int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t* out_profile,
+                    int32_t* out_free, int32_t* out_status, void* stream);
+
+/*
+ * Launch shape override for moc_eval_batch, for tuning.  threads_per_sequence is the number of
+ * threads that cooperate on one sequence (32, 64, 128, 256, 512 or 1024; 0 = choose from the
+ * graph size), sequences_per_block how many sequences one thread block works on at a time
+ * (0 = choose).  Results never depend on it.  MOC_ERR_ARG for unsupported values.
+ */
+int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t sequences_per_block);
+
+/* Number of kernels the most recent moc_eval_batch / moc_mem_profile on this thread launched. */
+int moc_last_launch_count(void);
+
+/* Text of the most recent error on the calling thread ("" if none). Owned by the library. */
+const char* moc_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOC_H_ */

@@ -1,0 +1,225 @@
+"""Thin ctypes binding of libmoc_b200.so (argument marshalling only; see include/moc.h).
+
+Function names mirror the C ABI.  PyTorch supplies device memory and streams: tensors are passed as
+``data_ptr()`` and the stream as ``torch.cuda.current_stream().cuda_stream``.  If the CUDA library
+has not been built, importing this module raises -- there is no CPU path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoc_b200.so")
+
+MOC_OK = 0
+ERROR_NAMES = {-1: "MOC_ERR_ARG", -2: "MOC_ERR_RANGE", -3: "MOC_ERR_CYCLE", -4: "MOC_ERR_OVERFLOW",
+               -5: "MOC_ERR_CUDA", -6: "MOC_ERR_NOMEM"}
+EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", "moc_graph_info",
+           "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
+           "moc_last_launch_count", "moc_last_error"]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
+                      "(nvcc, sm_100a). There is no CPU fallback.")
+
+lib = ctypes.CDLL(LIB_PATH)
+_P, _i32, _i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+lib.moc_graph_create.restype = ctypes.c_int
+lib.moc_graph_create.argtypes = [_i32, _i64, _P, _P, _P, ctypes.POINTER(_P)]
+lib.moc_graph_set_max_copies.restype = ctypes.c_int
+lib.moc_graph_set_max_copies.argtypes = [_P, _i32]
+lib.moc_graph_destroy.restype = None
+lib.moc_graph_destroy.argtypes = [_P]
+lib.moc_graph_info.restype = ctypes.c_int
+lib.moc_graph_info.argtypes = [_P, _P, _P, _P, _P]
+lib.moc_eval_batch.restype = ctypes.c_int
+lib.moc_eval_batch.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_eval_batch_host.restype = ctypes.c_int
+lib.moc_eval_batch_host.argtypes = [_P, _P, _i64, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_mem_profile.restype = ctypes.c_int
+lib.moc_mem_profile.argtypes = [_P, _P, _i32, _P, _P, _P, _P]
+lib.moc_graph_set_launch.restype = ctypes.c_int
+lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
+lib.moc_last_launch_count.restype = ctypes.c_int
+lib.moc_last_launch_count.argtypes = []
+lib.moc_last_error.restype = ctypes.c_char_p
+lib.moc_last_error.argtypes = []
+
+
+class MocError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        text = lib.moc_last_error().decode(errors="replace")
+        super().__init__(f"{where}: {ERROR_NAMES.get(code, code)}: {text}")
+
+
+def _check(rc, where):
+    if rc != MOC_OK:
+        raise MocError(rc, where)
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t, dtype, name):
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host(a, dtype, name):
+    """numpy array or CPU torch tensor -> pointer (the object must stay alive during the call)."""
+    import numpy as np
+    try:
+        import torch
+        if isinstance(a, torch.Tensor):
+            if a.is_cuda or not a.is_contiguous():
+                raise TypeError(f"{name}: expected a contiguous CPU tensor")
+            if a.numpy().dtype != np.dtype(dtype):
+                raise TypeError(f"{name}: expected dtype {dtype}")
+            return ctypes.c_void_p(a.data_ptr())
+    except ImportError:
+        pass
+    if not (isinstance(a, np.ndarray) and a.dtype == np.dtype(dtype) and a.flags.c_contiguous):
+        raise TypeError(f"{name}: expected a C-contiguous numpy array of {dtype}")
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def budget_from_peak(peak: int, pct: int) -> int:
+    """M = floor(peak * pct / 100): a budget given as a percentage of a no-rematerialization peak
+    (Section 4.3; the budgets printed there equal this rounding of a common integer peak)."""
+    return int(peak) * int(pct) // 100
+
+
+def moc_graph_create(n, edges, w, m):
+    """edges: (k, 2) int32 host array of (u, v) = v consumes u; w, m: int64 host arrays of n."""
+    import numpy as np
+    edges = np.ascontiguousarray(np.asarray(edges, np.int32).reshape(-1, 2))
+    w = np.ascontiguousarray(w, np.int64)
+    m = np.ascontiguousarray(m, np.int64)
+    if w.shape != (n,) or m.shape != (n,):
+        raise ValueError("w and m must have n entries")
+    h = _P()
+    rc = lib.moc_graph_create(int(n), len(edges), edges.ctypes.data if len(edges) else None,
+                              w.ctypes.data, m.ctypes.data, ctypes.byref(h))
+    _check(rc, "moc_graph_create")
+    return h
+
+
+def moc_graph_set_max_copies(g, C):
+    _check(lib.moc_graph_set_max_copies(g, int(C)), "moc_graph_set_max_copies")
+
+
+def moc_graph_set_launch(g, threads_per_sequence=0, sequences_per_block=0):
+    _check(lib.moc_graph_set_launch(g, int(threads_per_sequence), int(sequences_per_block)),
+           "moc_graph_set_launch")
+
+
+def moc_graph_destroy(g):
+    lib.moc_graph_destroy(g)
+
+
+def moc_graph_info(g):
+    n, ne, C, wide = _i32(), _i64(), _i32(), _i32()
+    _check(lib.moc_graph_info(g, ctypes.byref(n), ctypes.byref(ne), ctypes.byref(C), ctypes.byref(wide)),
+           "moc_graph_info")
+    return dict(n=n.value, n_edges=ne.value, C=C.value, wide=bool(wide.value))
+
+
+def moc_eval_batch(g, seqs, lens, M, out_peak=None, out_dur=None, out_feasible=None):
+    """Device tensors in, device tensors out (allocated with torch if not given). Asynchronous."""
+    import torch
+    B = lens.numel()
+    if out_peak is None:
+        out_peak = torch.empty(B, dtype=torch.int64, device=lens.device)
+    if out_dur is None:
+        out_dur = torch.empty(B, dtype=torch.int64, device=lens.device)
+    if out_feasible is None:
+        out_feasible = torch.empty(B, dtype=torch.int32, device=lens.device)
+    rc = lib.moc_eval_batch(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"), B, int(M),
+                            _dev(out_peak, torch.int64, "out_peak"), _dev(out_dur, torch.int64, "out_dur"),
+                            _dev(out_feasible, torch.int32, "out_feasible"), _stream())
+    _check(rc, "moc_eval_batch")
+    return out_peak, out_dur, out_feasible
+
+
+def moc_eval_batch_host(g, seqs, lens, M, out_peak, out_dur, out_feasible):
+    """Host arrays (numpy or CPU tensors, ideally pinned) in and out; returns after the results landed."""
+    import numpy as np
+    B = int(lens.shape[0])
+    rc = lib.moc_eval_batch_host(g, _host(seqs, np.int32, "seqs"), int(seqs.shape[0]), _host(lens, np.int32, "lens"),
+                                 B, int(M), _host(out_peak, np.int64, "out_peak"), _host(out_dur, np.int64, "out_dur"),
+                                 _host(out_feasible, np.int32, "out_feasible"), _stream())
+    _check(rc, "moc_eval_batch_host")
+    return out_peak, out_dur, out_feasible
+
+
+def moc_mem_profile(g, seq, want_free=True):
+    """One device sequence -> (profile[int64], free[int32] or None, status[int32 tensor of 1])."""
+    import torch
+    T = seq.numel()
+    profile = torch.empty(T, dtype=torch.int64, device=seq.device)
+    free = torch.empty(T, dtype=torch.int32, device=seq.device) if want_free else None
+    status = torch.empty(1, dtype=torch.int32, device=seq.device)
+    rc = lib.moc_mem_profile(g, _dev(seq, torch.int32, "seq"), T, _dev(profile, torch.int64, "profile"),
+                             _dev(free, torch.int32, "free") if want_free else None,
+                             _dev(status, torch.int32, "status"), _stream())
+    _check(rc, "moc_mem_profile")
+    return profile, free, status
+
+
+def moc_last_launch_count():
+    return lib.moc_last_launch_count()
+
+
+class Graph:
+    """Owns a moc_graph handle (created on the current CUDA device)."""
+
+    def __init__(self, n, edges, w, m, C=2):
+        self.n = int(n)
+        self.h = moc_graph_create(n, edges, w, m)
+        try:
+            moc_graph_set_max_copies(self.h, C)
+        except Exception:
+            moc_graph_destroy(self.h)
+            self.h = None
+            raise
+        self.C = int(C)
+
+    def close(self):
+        if getattr(self, "h", None):
+            moc_graph_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def info(self):
+        return moc_graph_info(self.h)
+
+    def set_launch(self, threads_per_sequence=0, sequences_per_block=0):
+        moc_graph_set_launch(self.h, threads_per_sequence, sequences_per_block)
+
+    def eval_batch(self, seqs, lens, M, **out):
+        return moc_eval_batch(self.h, seqs, lens, M, **out)
+
+    def eval_batch_host(self, seqs, lens, M, out_peak, out_dur, out_feasible):
+        return moc_eval_batch_host(self.h, seqs, lens, M, out_peak, out_dur, out_feasible)
+
+    def mem_profile(self, seq, want_free=True):
+        return moc_mem_profile(self.h, seq, want_free)
+
+    def no_remat_peak(self):
+        """Peak of the identity order 0..n-1 (the input topological order when ids are topological),
+        the reference point for budgets given in percent (Section 4.3)."""
+        import torch
+        seq = torch.arange(self.n, dtype=torch.int32, device="cuda")
+        lens = torch.tensor([self.n], dtype=torch.int32, device="cuda")
+        peak, _, st = self.eval_batch(seq, lens, (1 << 62))
+        torch.cuda.synchronize()
+        if int(st[0]) != 1:
+            raise ValueError("identity order is not a topological order of this graph")
+        return int(peak[0])

@@ -1,0 +1,485 @@
+// Host side of libmoc_b200.so: graph handle, validation, launch planning and the C ABI declared in
+// include/moc.h.  Every step of the evaluation itself runs in the kernels of moc_kernels.cuh.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/moc.h"
+#include "moc_kernels.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+thread_local int g_launches = 0;
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define MOC_CUDA(call)                                                                      \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return fail(e_ == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA,     \
+                        "%s: %s", #call, cudaGetErrorString(e_));                           \
+    } while (0)
+
+using KernelFn = void (*)(const moc::EvalParams);
+
+struct Plan {
+    bool valid = false;
+    KernelFn fn = nullptr;
+    int G = 0, gpc = 0, grid = 0, block = 0, CP = 0;
+    size_t smem = 0;
+    bool global_state = false, wide = false;
+    uint32_t cnt_bytes = 0, occ_bytes = 0, delta_bytes = 0, group_bytes = 0;
+};
+
+}  // namespace
+
+struct moc_graph {
+    int32_t n = 0;
+    int64_t n_edges = 0;  // distinct
+    int32_t C = 2;
+    int device = 0;
+    int sm_count = 0;
+    size_t smem_optin = 0;
+    int64_t sum_m = 0, sum_w = 0;
+    int32_t* d_succ_start = nullptr;
+    int32_t* d_succ = nullptr;
+    int64_t* d_w = nullptr;
+    int64_t* d_m64 = nullptr;
+    int32_t* d_m32 = nullptr;
+    int32_t want_G = 0, want_gpc = 0;
+    // grow-only scratch; mutable because evaluation takes a const handle
+    mutable Plan plan_eval, plan_profile;
+    mutable int64_t* d_offs = nullptr;
+    mutable size_t offs_cap = 0;
+    mutable char* d_state = nullptr;
+    mutable size_t state_cap = 0;
+    mutable int32_t* d_stage_seqs = nullptr;
+    mutable size_t stage_seqs_cap = 0;
+    mutable char* d_stage_io = nullptr;  // lens | peak | dur | status
+    mutable size_t stage_io_cap = 0;
+};
+
+namespace {
+
+size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
+
+template <int G, typename MemT>
+KernelFn shared_fn_cp(int CP, bool profile) {
+    if (profile && G != 1024) return nullptr;
+    switch (CP) {
+        case 2: return profile ? (KernelFn)moc::eval_shared_kernel<1024, MemT, 2, true>
+                               : (KernelFn)moc::eval_shared_kernel<G, MemT, 2, false>;
+        case 4: return profile ? (KernelFn)moc::eval_shared_kernel<1024, MemT, 4, true>
+                               : (KernelFn)moc::eval_shared_kernel<G, MemT, 4, false>;
+        default: return profile ? (KernelFn)moc::eval_shared_kernel<1024, MemT, 8, true>
+                                : (KernelFn)moc::eval_shared_kernel<G, MemT, 8, false>;
+    }
+}
+template <typename MemT>
+KernelFn shared_fn_g(int G, int CP, bool profile) {
+    switch (G) {
+        case 32: return shared_fn_cp<32, MemT>(CP, profile);
+        case 64: return shared_fn_cp<64, MemT>(CP, profile);
+        case 128: return shared_fn_cp<128, MemT>(CP, profile);
+        case 256: return shared_fn_cp<256, MemT>(CP, profile);
+        case 512: return shared_fn_cp<512, MemT>(CP, profile);
+        case 1024: return shared_fn_cp<1024, MemT>(CP, profile);
+        default: return nullptr;
+    }
+}
+KernelFn global_fn(int CP, bool profile) {
+    switch (CP) {
+        case 2: return profile ? (KernelFn)moc::eval_global_kernel<2, true> : (KernelFn)moc::eval_global_kernel<2, false>;
+        case 4: return profile ? (KernelFn)moc::eval_global_kernel<4, true> : (KernelFn)moc::eval_global_kernel<4, false>;
+        default: return profile ? (KernelFn)moc::eval_global_kernel<8, true> : (KernelFn)moc::eval_global_kernel<8, false>;
+    }
+}
+
+int pow2_ceil(int x) {
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+// Chooses kernel variant, group size and grid for the handle's current n and C.
+int make_plan(const moc_graph* g, bool profile, Plan* out) {
+    Plan pl;
+    const int64_t n = g->n, C = g->C;
+    pl.CP = C <= 2 ? 2 : (C <= 4 ? 4 : 8);
+    pl.wide = g->sum_m > (int64_t)INT32_MAX / C;  // C*sum(m) bounds every partial sum of deltas
+    const int64_t t_max = C * n;
+    const size_t mem_sz = pl.wide ? 8 : 4;
+    const size_t sh_cnt = align16(4 * n), sh_occ = align16(2 * n * pl.CP),
+                 sh_delta = align16((t_max + 1) * mem_sz);
+    const size_t sh_group = sh_cnt + sh_occ + sh_delta + align16(moc::kRedBytes);
+    const size_t smem_cap = g->smem_optin > 1024 ? g->smem_optin - 1024 : 0;  // 1 KB per block is reserved
+    if (t_max <= 65534 && sh_group <= smem_cap) {
+        pl.global_state = false;
+        pl.cnt_bytes = (uint32_t)sh_cnt;
+        pl.occ_bytes = (uint32_t)sh_occ;
+        pl.delta_bytes = (uint32_t)sh_delta;
+        pl.group_bytes = (uint32_t)sh_group;
+        int G = 1024, gpc = 1;
+        if (!profile) {
+            const int per_sm = (int)std::max<size_t>(1, g->smem_optin / sh_group);  // groups resident per SM
+            G = g->want_G ? g->want_G : std::min(1024, std::max(32, pow2_ceil(32 * 48 / std::min(per_sm, 48))));
+            gpc = g->want_gpc ? g->want_gpc : std::max(1, 256 / G);
+            gpc = std::min(gpc, G == 32 ? 32 : 15);          // named barriers 1..15
+            gpc = std::min(gpc, 1024 / G);
+            while (gpc > 1 && (size_t)gpc * sh_group > smem_cap) --gpc;
+        }
+        pl.G = G;
+        pl.gpc = gpc;
+        pl.block = G * gpc;
+        pl.smem = (size_t)gpc * sh_group;
+        pl.fn = pl.wide ? shared_fn_g<int64_t>(G, pl.CP, profile) : shared_fn_g<int32_t>(G, pl.CP, profile);
+        if (!pl.fn) return fail(MOC_ERR_ARG, "unsupported launch shape");
+        cudaError_t e = cudaFuncSetAttribute((const void*)pl.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+        if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        int nb = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)pl.fn, pl.block, pl.smem);
+        if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "occupancy query: %s", cudaGetErrorString(e));
+        if (nb < 1) return fail(MOC_ERR_CUDA, "kernel does not fit on an SM (block %d, smem %zu)", pl.block, pl.smem);
+        pl.grid = profile ? 1 : g->sm_count * nb;
+    } else {
+        // state in global memory: int32 positions, int64 sums
+        pl.global_state = true;
+        pl.wide = true;
+        pl.cnt_bytes = (uint32_t)align16(4 * n);
+        const size_t occ = align16(4 * n * pl.CP), del = align16((t_max + 1) * 8);
+        const size_t grp = pl.cnt_bytes + occ + del + align16(moc::kRedBytes);
+        if (grp > 0xFFFFFFFFull) return fail(MOC_ERR_ARG, "graph too large: per-sequence state of %zu bytes", grp);
+        pl.occ_bytes = (uint32_t)occ;
+        pl.delta_bytes = (uint32_t)del;
+        pl.group_bytes = (uint32_t)grp;
+        pl.G = 1024;
+        pl.gpc = 1;
+        pl.block = 1024;
+        pl.smem = 0;
+        pl.fn = global_fn(pl.CP, profile);
+        int nb = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)pl.fn, pl.block, 0);
+        if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "occupancy query: %s", cudaGetErrorString(e));
+        if (nb < 1) nb = 1;
+        pl.grid = profile ? 1 : g->sm_count * nb;
+    }
+    pl.valid = true;
+    *out = pl;
+    return MOC_OK;
+}
+
+int ensure(void** ptr, size_t* cap, size_t need) {
+    if (need <= *cap) return MOC_OK;
+    if (*ptr) {
+        MOC_CUDA(cudaFree(*ptr));
+        *ptr = nullptr;
+        *cap = 0;
+    }
+    size_t want = std::max(need, *cap * 2);
+    MOC_CUDA(cudaMalloc(ptr, want));
+    *cap = want;
+    return MOC_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
+    moc::EvalParams p{};
+    p.g.n = g->n;
+    p.g.C = g->C;
+    p.g.succ_start = g->d_succ_start;
+    p.g.succ = g->d_succ;
+    p.g.w = g->d_w;
+    p.g.m = pl.wide ? (const void*)g->d_m64 : (const void*)g->d_m32;
+    p.cnt_bytes = pl.cnt_bytes;
+    p.occ_bytes = pl.occ_bytes;
+    p.delta_bytes = pl.delta_bytes;
+    p.group_bytes = pl.group_bytes;
+    return p;
+}
+
+int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B, int64_t M,
+                int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st) {
+    if (!g->plan_eval.valid) {
+        int rc = make_plan(g, false, &g->plan_eval);
+        if (rc != MOC_OK) return rc;
+    }
+    const Plan& pl = g->plan_eval;
+    int rc = ensure((void**)&g->d_offs, &g->offs_cap, ((size_t)B + 1) * sizeof(int64_t));
+    if (rc != MOC_OK) return rc;
+    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    if (pl.global_state) {
+        rc = ensure((void**)&g->d_state, &g->state_cap, (size_t)pl.grid * pl.group_bytes);
+        if (rc != MOC_OK) return rc;
+    }
+    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, g->d_offs);
+    ++g_launches;
+    moc::EvalParams p = base_params(g, pl);
+    p.seqs = seqs;
+    p.lens = lens;
+    p.offs = g->d_offs;
+    p.B = B;
+    p.M = M;
+    p.out_peak = out_peak;
+    p.out_dur = out_dur;
+    p.out_status = out_feasible;
+    p.gstate = g->d_state;
+    pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
+    ++g_launches;
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moc_last_error(void) { return g_err; }
+int moc_last_launch_count(void) { return g_launches; }
+
+int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int64_t* w,
+                     const int64_t* m, moc_graph** out) {
+    g_err[0] = 0;
+    if (out) *out = nullptr;
+    if (!out || !w || !m || n < 1 || n_edges < 0 || (n_edges > 0 && !edges))
+        return fail(MOC_ERR_ARG, "moc_graph_create: null pointer, n < 1 or n_edges < 0");
+    if (n > (1 << 27) || n_edges > (int64_t)INT32_MAX - 1)
+        return fail(MOC_ERR_ARG, "moc_graph_create: n > 2^27 or n_edges >= 2^31-1");
+    int64_t sum_w = 0, sum_m = 0;
+    const int64_t lim = (int64_t(1) << 62) / 8;
+    for (int32_t v = 0; v < n; ++v) {
+        if (w[v] < 0 || m[v] < 0) return fail(MOC_ERR_OVERFLOW, "negative weight at node %d", v);
+        if (w[v] >= lim - sum_w || m[v] >= lim - sum_m)
+            return fail(MOC_ERR_OVERFLOW, "8*sum(w) or 8*sum(m) reaches 2^62");
+        sum_w += w[v];
+        sum_m += m[v];
+    }
+    std::vector<uint64_t> keys;
+    try {
+        keys.reserve((size_t)n_edges);
+        for (int64_t e = 0; e < n_edges; ++e) {
+            const int32_t u = edges[2 * e], v = edges[2 * e + 1];
+            if (u < 0 || u >= n || v < 0 || v >= n)
+                return fail(MOC_ERR_RANGE, "edge %lld = (%d,%d) outside [0,%d)", (long long)e, u, v, n);
+            if (u == v) return fail(MOC_ERR_CYCLE, "self-loop at node %d", u);
+            keys.push_back(((uint64_t)(uint32_t)u << 32) | (uint32_t)v);
+        }
+        std::sort(keys.begin(), keys.end());
+        keys.erase(std::unique(keys.begin(), keys.end()), keys.end());
+    } catch (const std::bad_alloc&) {
+        return fail(MOC_ERR_NOMEM, "host allocation failed");
+    }
+    const int64_t ne = (int64_t)keys.size();
+    std::vector<int32_t> succ_start, succ, indeg, queue, m32;
+    try {
+        succ_start.assign((size_t)n + 1, 0);
+        succ.resize((size_t)std::max<int64_t>(ne, 1));
+        indeg.assign((size_t)n, 0);
+        m32.resize((size_t)n);
+        for (int64_t e = 0; e < ne; ++e) {
+            const int32_t u = (int32_t)(keys[e] >> 32), v = (int32_t)(keys[e] & 0xFFFFFFFFu);
+            succ_start[u + 1]++;
+            succ[e] = v;  // keys are sorted by (u, v): already grouped by producer
+            indeg[v]++;
+        }
+        for (int32_t v = 0; v < n; ++v) succ_start[v + 1] += succ_start[v];
+        // Kahn: the graph is a DAG iff every node gets removed
+        queue.reserve((size_t)n);
+        for (int32_t v = 0; v < n; ++v)
+            if (indeg[v] == 0) queue.push_back(v);
+        for (size_t h = 0; h < queue.size(); ++h) {
+            const int32_t u = queue[h];
+            for (int32_t e = succ_start[u]; e < succ_start[u + 1]; ++e)
+                if (--indeg[succ[e]] == 0) queue.push_back(succ[e]);
+        }
+        if ((int32_t)queue.size() != n) return fail(MOC_ERR_CYCLE, "the edges contain a directed cycle");
+        for (int32_t v = 0; v < n; ++v) m32[v] = (int32_t)std::min<int64_t>(m[v], INT32_MAX);
+    } catch (const std::bad_alloc&) {
+        return fail(MOC_ERR_NOMEM, "host allocation failed");
+    }
+
+    moc_graph* g = new (std::nothrow) moc_graph();
+    if (!g) return fail(MOC_ERR_NOMEM, "host allocation failed");
+    g->n = n;
+    g->n_edges = ne;
+    g->sum_m = sum_m;
+    g->sum_w = sum_w;
+    int rc = MOC_OK;
+    cudaError_t e = cudaGetDevice(&g->device);
+    int smem = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, g->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, g->device);
+    g->smem_optin = (size_t)smem;
+    auto up = [&](void** dst, const void* src, size_t bytes) {
+        if (e != cudaSuccess) return;
+        e = cudaMalloc(dst, std::max<size_t>(bytes, 16));
+        if (e == cudaSuccess && bytes) e = cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice);
+    };
+    up((void**)&g->d_succ_start, succ_start.data(), ((size_t)n + 1) * 4);
+    up((void**)&g->d_succ, succ.data(), (size_t)ne * 4);
+    up((void**)&g->d_w, w, (size_t)n * 8);
+    up((void**)&g->d_m64, m, (size_t)n * 8);
+    up((void**)&g->d_m32, m32.data(), (size_t)n * 4);
+    if (e != cudaSuccess) {
+        rc = fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA,
+                  "moc_graph_create: %s", cudaGetErrorString(e));
+        cudaGetLastError();
+        moc_graph_destroy(g);
+        return rc;
+    }
+    *out = g;
+    return MOC_OK;
+}
+
+int moc_graph_set_max_copies(moc_graph* g, int32_t C) {
+    g_err[0] = 0;
+    if (!g || C < 1 || C > MOC_MAX_COPIES) return fail(MOC_ERR_ARG, "moc_graph_set_max_copies: C must be 1..%d", MOC_MAX_COPIES);
+    g->C = C;
+    g->plan_eval.valid = false;
+    g->plan_profile.valid = false;
+    return MOC_OK;
+}
+
+int moc_graph_set_launch(moc_graph* g, int32_t tps, int32_t spb) {
+    g_err[0] = 0;
+    const bool ok_g = tps == 0 || tps == 32 || tps == 64 || tps == 128 || tps == 256 || tps == 512 || tps == 1024;
+    if (!g || !ok_g || spb < 0 || spb > 32 || (tps && spb && tps * spb > 1024))
+        return fail(MOC_ERR_ARG, "moc_graph_set_launch: unsupported shape (%d threads x %d sequences)", tps, spb);
+    g->want_G = tps;
+    g->want_gpc = spb;
+    g->plan_eval.valid = false;
+    return MOC_OK;
+}
+
+void moc_graph_destroy(moc_graph* g) {
+    if (!g) return;
+    DeviceGuard dg(g->device);
+    cudaFree(g->d_succ_start);
+    cudaFree(g->d_succ);
+    cudaFree(g->d_w);
+    cudaFree(g->d_m64);
+    cudaFree(g->d_m32);
+    cudaFree(g->d_offs);
+    cudaFree(g->d_state);
+    cudaFree(g->d_stage_seqs);
+    cudaFree(g->d_stage_io);
+    delete g;
+}
+
+int moc_graph_info(const moc_graph* g, int32_t* n, int64_t* n_edges, int32_t* C, int32_t* wide) {
+    g_err[0] = 0;
+    if (!g) return fail(MOC_ERR_ARG, "moc_graph_info: null handle");
+    if (n) *n = g->n;
+    if (n_edges) *n_edges = g->n_edges;
+    if (C) *C = g->C;
+    if (wide) *wide = g->sum_m > (int64_t)INT32_MAX / g->C ? 1 : 0;
+    return MOC_OK;
+}
+
+int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B, int64_t M,
+                   int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, void* stream) {
+    g_err[0] = 0;
+    g_launches = 0;
+    if (!g || B < 0) return fail(MOC_ERR_ARG, "moc_eval_batch: null handle or B < 0");
+    if (B == 0) return MOC_OK;
+    if (!seqs || !lens || !out_peak || !out_dur || !out_feasible)
+        return fail(MOC_ERR_ARG, "moc_eval_batch: null array");
+    if (reinterpret_cast<uintptr_t>(seqs) & 3) return fail(MOC_ERR_ARG, "moc_eval_batch: seqs not 4-byte aligned");
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    return launch_eval(g, seqs, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream);
+}
+
+int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps, const int32_t* lens,
+                        int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur,
+                        int32_t* out_feasible, void* stream) {
+    g_err[0] = 0;
+    g_launches = 0;
+    if (!g || B < 0 || n_steps < 0) return fail(MOC_ERR_ARG, "moc_eval_batch_host: null handle or negative size");
+    if (B == 0) return MOC_OK;
+    if (!lens || !out_peak || !out_dur || !out_feasible || (n_steps > 0 && !seqs))
+        return fail(MOC_ERR_ARG, "moc_eval_batch_host: null array");
+    int64_t need = 0;
+    for (int32_t b = 0; b < B; ++b) need += lens[b] > 0 ? lens[b] : 0;
+    if (need > n_steps) return fail(MOC_ERR_ARG, "moc_eval_batch_host: lens sum to %lld > n_steps %lld", (long long)need, (long long)n_steps);
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = ensure((void**)&g->d_stage_seqs, &g->stage_seqs_cap, std::max<size_t>((size_t)need * 4, 16));
+    if (rc != MOC_OK) return rc;
+    const size_t bB = (size_t)B, o_lens = 0, o_peak = align16(bB * 4), o_dur = o_peak + bB * 8,
+                 o_st = o_dur + bB * 8, io_bytes = o_st + bB * 4;
+    rc = ensure((void**)&g->d_stage_io, &g->stage_io_cap, io_bytes);
+    if (rc != MOC_OK) return rc;
+    int32_t* d_lens = (int32_t*)(g->d_stage_io + o_lens);
+    int64_t* d_peak = (int64_t*)(g->d_stage_io + o_peak);
+    int64_t* d_dur = (int64_t*)(g->d_stage_io + o_dur);
+    int32_t* d_st = (int32_t*)(g->d_stage_io + o_st);
+    if (need) MOC_CUDA(cudaMemcpyAsync(g->d_stage_seqs, seqs, (size_t)need * 4, cudaMemcpyHostToDevice, st));
+    MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, st));
+    rc = launch_eval(g, g->d_stage_seqs, d_lens, B, M, d_peak, d_dur, d_st, st);
+    if (rc != MOC_OK) return rc;
+    MOC_CUDA(cudaMemcpyAsync(out_peak, d_peak, bB * 8, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaMemcpyAsync(out_dur, d_dur, bB * 8, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaMemcpyAsync(out_feasible, d_st, bB * 4, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaStreamSynchronize(st));
+    return MOC_OK;
+}
+
+int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t* out_profile,
+                    int32_t* out_free, int32_t* out_status, void* stream) {
+    g_err[0] = 0;
+    g_launches = 0;
+    if (!g || len < 0 || !out_status || (len > 0 && (!seq || !out_profile)))
+        return fail(MOC_ERR_ARG, "moc_mem_profile: null pointer or len < 0");
+    if (reinterpret_cast<uintptr_t>(seq) & 3) return fail(MOC_ERR_ARG, "moc_mem_profile: seq not 4-byte aligned");
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!g->plan_profile.valid) {
+        int rc = make_plan(g, true, &g->plan_profile);
+        if (rc != MOC_OK) return rc;
+    }
+    const Plan& pl = g->plan_profile;
+    if (pl.global_state) {
+        int rc = ensure((void**)&g->d_state, &g->state_cap, (size_t)pl.group_bytes);
+        if (rc != MOC_OK) return rc;
+    }
+    moc::EvalParams p = base_params(g, pl);
+    p.seqs = seq;
+    p.single_len = len;
+    p.B = 1;
+    p.M = INT64_MAX;
+    p.out_status = out_status;
+    p.out_profile = out_profile;
+    p.out_free = out_free;
+    p.gstate = g->d_state;
+    pl.fn<<<1, pl.block, pl.smem, st>>>(p);
+    ++g_launches;
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+
+}  // extern "C"

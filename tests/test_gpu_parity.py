@@ -1,0 +1,271 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact on peak, duration,
+status, and -- for moc_mem_profile -- on every profile entry and free step."""
+import numpy as np
+import pytest
+import torch
+
+import pins
+from oracle import OracleGraph
+from paper_2304_14463_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+BIG = 1 << 60
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2304_14463_b200 import build
+    build.build()
+    from paper_2304_14463_b200 import binding
+    return binding
+
+
+def dev(a, dtype=torch.int32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype).cuda()
+
+
+def gpu_eval(G, seqs, lens, M):
+    peak, dur, st = G.eval_batch(dev(seqs), dev(lens), M)
+    torch.cuda.synchronize()
+    return peak.cpu().numpy(), dur.cpu().numpy(), st.cpu().numpy()
+
+
+def assert_batch_equal(G, O, seqs, lens, M, what=""):
+    gp, gd, gs = gpu_eval(G, seqs, lens, M)
+    op, od, os_, _ = O.eval_batch(seqs, lens, M, n_threads=4)
+    bad = np.nonzero((gp != op) | (gd != od) | (gs != os_))[0]
+    assert len(bad) == 0, f"{what}: {len(bad)} of {len(lens)} differ, first {bad[:5]}: gpu " \
+                          f"{gp[bad[:3]], gd[bad[:3]], gs[bad[:3]]} oracle {op[bad[:3]], od[bad[:3]], os_[bad[:3]]}"
+    return op, od, os_
+
+
+# ------------------------------------------------------------------ the oracle's pins, on the GPU
+def test_pins_through_the_gpu(B):
+    class GpuGraph:
+        def __init__(self, n, edges, w, m, C):
+            self.G = B.Graph(n, edges, w, m, C)
+
+        def eval(self, seq, M):
+            seq = np.asarray(seq, np.int32)
+            p, d, s = gpu_eval(self.G, seq, np.array([len(seq)], np.int32), M)
+            prof, free, st = self.G.mem_profile(dev(seq))
+            torch.cuda.synchronize()
+            assert (int(st[0]) < 0) == (int(s[0]) < 0) and (int(s[0]) >= 0 or int(st[0]) == int(s[0]))
+            return dict(peak=int(p[0]), dur=int(d[0]), status=int(s[0]),
+                        profile=prof.cpu().numpy(), free=free.cpu().numpy())
+
+    for pin in (pins.pin_paper_example, pins.pin_small_cases, pins.pin_random_remat):
+        pin(lambda n, e, w, m, C: GpuGraph(n, e, w, m, C))
+
+
+# ------------------------------------------------------------------ the five configurations
+SMALL_B = [1024, 4096, 2048, 512, 64]
+
+
+@pytest.mark.parametrize("idx", range(W.N_CONFIGS))
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_config_parity_mutated(B, idx, seed):
+    """Reduced batches, 1/16 of the sequences damaged, budgets that make both 0 and 1 occur."""
+    wl = W.make(idx, seed=seed, B=SMALL_B[idx])
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    P0 = O.eval(np.arange(wl.n), BIG)["peak"]
+    assert G.no_remat_peak() == P0
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=seed, frac=1 / 16)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    median = int(np.median(peaks[peaks >= 0]))
+    seen = set()
+    for M in [B.budget_from_peak(P0, p) for p in wl.budget_pcts] + [P0, median]:
+        _, _, st = assert_batch_equal(G, O, seqs, lens, M, f"{wl.name} seed {seed} M {M}")
+        seen |= set(np.unique(st).tolist())
+    assert {-2, 0, 1} <= seen and (idx == 4 or -1 in seen)
+
+
+@pytest.mark.parametrize("idx", range(W.N_CONFIGS))
+def test_config_parity_full_size(B, idx):
+    """The full batch of every configuration in the launch shape the benchmark times."""
+    wl = W.make(idx, seed=1)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    P0 = G.no_remat_peak()
+    for pct in wl.budget_pcts:
+        assert_batch_equal(G, O, wl.seqs, wl.lens, B.budget_from_peak(P0, pct), f"{wl.name} {pct}%")
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
+def test_wide_arithmetic(B, idx):
+    """Output sizes scaled so that sums need 64 bits."""
+    wl = W.make(idx, seed=4, B=min(SMALL_B[idx], 256))
+    m = wl.m * (1 << 24) + 12345
+    O = OracleGraph(wl.n, wl.edges, wl.w * (1 << 30), m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w * (1 << 30), m, wl.C)
+    assert G.info()["wide"]
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=9, frac=1 / 8)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    assert peaks.max() > (1 << 32)
+    assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), wl.name)
+
+
+@pytest.mark.parametrize("idx", [0, 2, 3])
+def test_mem_profile_parity(B, idx):
+    wl = W.make(idx, seed=5, B=24)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=2, frac=0.3)
+    for seq in W.unpack(seqs, lens):
+        r = O.eval(seq, BIG)
+        prof, free, st = G.mem_profile(dev(seq))
+        torch.cuda.synchronize()
+        assert int(st[0]) == r["status"]
+        assert (prof.cpu().numpy() == r["profile"]).all() and (free.cpu().numpy() == r["free"]).all()
+    prof, free, st = G.mem_profile(dev(seq), want_free=False)
+    torch.cuda.synchronize()
+    assert free is None and (prof.cpu().numpy() == r["profile"]).all()
+
+
+# ------------------------------------------------------------------ launch shapes, alignment, edges
+@pytest.mark.parametrize("tps,spb", [(32, 1), (32, 8), (32, 16), (64, 4), (128, 2), (256, 1), (256, 3),
+                                     (512, 1), (512, 2), (1024, 1)])
+def test_every_launch_shape(B, tps, spb):
+    wl = W.make(2, seed=6, B=700)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G.set_launch(tps, spb)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=3, frac=1 / 8)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), f"shape {tps}x{spb}")
+
+
+@pytest.mark.parametrize("C", [1, 2, 3, 4, 5, 8])
+def test_every_copy_cap(B, C):
+    n = 150
+    edges = W.layered_dag(n, 400, 10, seed=C)
+    w = W.weights_uniform(n, 1, 9, 1, 1)
+    m = W.weights_lognormal(n, 5.0, 1.0, 1, 2)
+    seqs, lens = W.schedules(n, edges, C, 0.35, 300, seed=C)
+    seqs, lens = W.mutate(seqs, lens, n, C, seed=C, frac=1 / 8)
+    O = OracleGraph(n, edges, w, m, C)
+    G = B.Graph(n, edges, w, m, C)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), f"C={C}")
+    # the cap is what makes a sequence malformed: the same sequences under a smaller cap
+    if C > 1:
+        O2 = OracleGraph(n, edges, w, m, C - 1)
+        B.moc_graph_set_max_copies(G.h, C - 1)
+        assert_batch_equal(G, O2, seqs, lens, BIG, f"C={C} evaluated with cap {C - 1}")
+
+
+def test_unaligned_rows_and_views(B):
+    """Rows start at every 4-byte phase; the packed array itself starts off a 16-byte boundary."""
+    wl = W.make(1, seed=7, B=500)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    op, od, os_, _ = O.eval_batch(wl.seqs, wl.lens, BIG)
+    for shift in (1, 2, 3):
+        buf = torch.zeros(len(wl.seqs) + 8, dtype=torch.int32, device="cuda")
+        view = buf[shift:shift + len(wl.seqs)]
+        view.copy_(dev(wl.seqs))
+        assert view.data_ptr() % 16 == 4 * shift
+        peak, dur, st = G.eval_batch(view, dev(wl.lens), BIG)
+        torch.cuda.synchronize()
+        assert (peak.cpu().numpy() == op).all() and (dur.cpu().numpy() == od).all() and (st.cpu().numpy() == os_).all()
+
+
+def test_degenerate_batches(B):
+    n = 5
+    edges = [(0, 1), (1, 2), (0, 3)]
+    w = np.arange(1, 6)
+    m = np.array([5, 1, 2, 3, 4])
+    O = OracleGraph(n, edges, w, m, 2)
+    G = B.Graph(n, edges, w, m, 2)
+    # B = 0: nothing happens
+    e = torch.empty(0, dtype=torch.int32, device="cuda")
+    p, d, s = G.eval_batch(e, e, 10)
+    assert p.numel() == 0 and B.moc_last_launch_count() == 0
+    # zero, negative, too short, exactly n, exactly C*n, too long
+    rows = [[], [0, 1, 2], [0, 1, 2, 3, 4], [0, 0, 1, 1, 2, 2, 3, 3, 4, 4], [0, 1, 2, 3, 4] * 2 + [0], [4, 3, 2, 1, 0]]
+    seqs, lens = W.pack(rows)
+    lens = np.concatenate([lens, [-3]]).astype(np.int32)
+    assert_batch_equal(G, O, seqs, lens, 9, "degenerate")
+    # single isolated node
+    O1, G1 = OracleGraph(1, [], [7], [3], 2), B.Graph(1, [], [7], [3], 2)
+    seqs, lens = W.pack([[0], [0, 0], [0, 0, 0], [1]])
+    assert_batch_equal(G1, O1, seqs, lens, 3, "single node")
+    # duplicate edges are merged
+    G2 = B.Graph(n, edges + edges, w, m, 2)
+    assert G2.info()["n_edges"] == 3
+    # mem_profile of an empty and of a malformed sequence
+    prof, free, st = G.mem_profile(torch.empty(0, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(st[0]) == -2
+    prof, free, st = G.mem_profile(dev([0, 1, 2, 3, 9]))
+    torch.cuda.synchronize()
+    assert int(st[0]) == -2 and (prof.cpu().numpy() == -1).all() and (free.cpu().numpy() == -1).all()
+
+
+def test_determinism_and_reuse(B):
+    wl = W.make(2, seed=8, B=3000)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    s, l = dev(wl.seqs), dev(wl.lens)
+    a = [t.clone() for t in G.eval_batch(s, l, 12345678)]
+    for _ in range(3):
+        b = G.eval_batch(s, l, 12345678)
+        torch.cuda.synchronize()
+        assert all(torch.equal(x, y) for x, y in zip(a, b))
+    # a smaller batch after a larger one on the same handle
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    assert_batch_equal(G, O, wl.seqs[:int(wl.lens[:10].sum())], wl.lens[:10], BIG, "reuse")
+    assert B.moc_last_launch_count() == 2
+
+
+def test_host_entry_point(B):
+    wl = W.make(1, seed=9, B=2000)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs = torch.from_numpy(wl.seqs).pin_memory()
+    lens = torch.from_numpy(wl.lens).pin_memory()
+    peak = torch.empty(wl.B, dtype=torch.int64).pin_memory()
+    dur = torch.empty(wl.B, dtype=torch.int64).pin_memory()
+    st = torch.empty(wl.B, dtype=torch.int32).pin_memory()
+    M = 30000
+    G.eval_batch_host(seqs, lens, M, peak, dur, st)
+    op, od, os_, _ = O.eval_batch(wl.seqs, wl.lens, M)
+    assert (peak.numpy() == op).all() and (dur.numpy() == od).all() and (st.numpy() == os_).all()
+    # pageable numpy arrays work too
+    p2, d2, s2 = np.empty(wl.B, np.int64), np.empty(wl.B, np.int64), np.empty(wl.B, np.int32)
+    G.eval_batch_host(wl.seqs, wl.lens, M, p2, d2, s2)
+    assert (p2 == op).all() and (d2 == od).all() and (s2 == os_).all()
+
+
+def test_state_in_global_memory(B):
+    """A graph whose per-sequence state exceeds shared memory (and > 65534 steps per sequence)."""
+    n, C = 40000, 2
+    edges = W.layered_dag(n, 3 * n, 40, seed=3)
+    w = W.weights_uniform(n, 1, 100, 3, 1)
+    m = W.weights_lognormal(n, 8.0, 2.0, 3, 2)
+    seqs, lens = W.schedules(n, edges, C, 0.7, 6, seed=11)
+    assert lens.max() > 65534
+    seqs, lens = W.mutate(seqs, lens, n, C, seed=1, frac=0.34)
+    O = OracleGraph(n, edges, w, m, C)
+    G = B.Graph(n, edges, w, m, C)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), "global state")
+    seq = W.unpack(seqs, lens)[int(np.argmax(peaks >= 0))]
+    r = O.eval(seq, BIG)
+    prof, free, st = G.mem_profile(dev(seq))
+    torch.cuda.synchronize()
+    assert int(st[0]) == 1 and (prof.cpu().numpy() == r["profile"]).all() and (free.cpu().numpy() == r["free"]).all()
+
+
+def test_sampled_invariants_at_full_size(B):
+    """Properties that hold at any size, on the benchmark workload (no oracle involved)."""
+    wl = W.make(2, seed=1)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    peak, dur, st = gpu_eval(G, wl.seqs, wl.lens, BIG)
+    lower = wl.m.copy()
+    np.add.at(lower, wl.edges[:, 1], wl.m[wl.edges[:, 0]])
+    assert (st == 1).all() and (peak >= lower.max()).all()
+    offs = np.concatenate([[0], np.cumsum(wl.lens)])
+    wsum = np.add.reduceat(wl.w[wl.seqs], offs[:-1])
+    msum = np.add.reduceat(wl.m[wl.seqs], offs[:-1])
+    assert (dur == wsum).all() and (peak <= msum).all()
