@@ -190,9 +190,9 @@ class Graph:
             raise
         self.C = int(C)
 
-    def close(self):
+    def close(self, _destroy=lib.moc_graph_destroy):
         if getattr(self, "h", None):
-            moc_graph_destroy(self.h)
+            _destroy(self.h)
             self.h = None
 
     __del__ = close
