@@ -117,6 +117,37 @@ int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps
                         int64_t* out_dur, int32_t* out_feasible, void* stream);
 
 /*
+ * moc_eval_batch for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a deployment variant of moc_eval_batch, with identical results.)
+ *
+ * Who needs it: a caller that has handed the whole device to its own memory pool, a latency-bound
+ * loop that cannot afford the driver's allocator lock or the device-wide synchronisation that
+ * cudaFree implies, or a process running under a fixed memory partition.  moc_eval_batch keeps its
+ * packing offsets (B+1 int64) in scratch that it allocates on the handle and regrows when B grows;
+ * this entry point keeps them in a fixed array inside the library image instead, and calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   - The array holds MOC_NOALLOC_MAX_B + 1 offsets (512 KB).  It is part of the library's device
+ *     image: every GPU on which the library is used holds it until the process exits.
+ *   - B > MOC_NOALLOC_MAX_B is rejected with MOC_ERR_ARG.  So is a graph whose per-sequence state
+ *     does not fit in shared memory (more than 65534 steps per sequence, or n*C too large): that
+ *     case needs a global workspace, which only moc_eval_batch provides.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current) and prepares the launch plan of the handle.  Make that first call
+ *     outside of any stream capture.
+ *   - All calls on a device, from every handle and stream, share the one array.  Each call
+ *     rewrites the B+1 entries it uses before reading them, so stale contents of an earlier call
+ *     never matter and nothing needs clearing; but two calls that overlap on the GPU (different
+ *     streams without an ordering between them) race on it and give wrong results.  Order them.
+ *
+ * Arguments, outputs, asynchrony and status codes are exactly those of moc_eval_batch.
+ */
+#define MOC_NOALLOC_MAX_B 65536
+int moc_eval_batch_noalloc(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B,
+                           int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
+                           void* stream);
+
+/*
  * Memory profile of one sequence (the per-event sums of Eq. 4 and the interval ends of Section 2).
  *   seq          DEVICE, len int32 node ids.
  *   out_profile  DEVICE, len int64: memory in use at every step.

@@ -17,7 +17,7 @@ ERROR_NAMES = {-1: "MOC_ERR_ARG", -2: "MOC_ERR_RANGE", -3: "MOC_ERR_CYCLE", -4: 
                -5: "MOC_ERR_CUDA", -6: "MOC_ERR_NOMEM"}
 EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", "moc_graph_info",
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
-           "moc_last_launch_count", "moc_last_error"]
+           "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -37,6 +37,8 @@ lib.moc_eval_batch.restype = ctypes.c_int
 lib.moc_eval_batch.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_eval_batch_host.restype = ctypes.c_int
 lib.moc_eval_batch_host.argtypes = [_P, _P, _i64, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_eval_batch_noalloc.restype = ctypes.c_int
+lib.moc_eval_batch_noalloc.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_mem_profile.restype = ctypes.c_int
 lib.moc_mem_profile.argtypes = [_P, _P, _i32, _P, _P, _P, _P]
 lib.moc_graph_set_launch.restype = ctypes.c_int
@@ -144,6 +146,22 @@ def moc_eval_batch(g, seqs, lens, M, out_peak=None, out_dur=None, out_feasible=N
                             _dev(out_peak, torch.int64, "out_peak"), _dev(out_dur, torch.int64, "out_dur"),
                             _dev(out_feasible, torch.int32, "out_feasible"), _stream())
     _check(rc, "moc_eval_batch")
+    return out_peak, out_dur, out_feasible
+
+
+MOC_NOALLOC_MAX_B = 65536
+
+
+def moc_eval_batch_noalloc(g, seqs, lens, M, out_peak, out_dur, out_feasible):
+    """moc_eval_batch for callers that must not allocate: every tensor, outputs included, is passed
+    in, and the library keeps its packing offsets in a fixed array of its own device image (at most
+    MOC_NOALLOC_MAX_B sequences per call; calls on one device must not overlap on the GPU)."""
+    import torch
+    rc = lib.moc_eval_batch_noalloc(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"),
+                                    lens.numel(), int(M), _dev(out_peak, torch.int64, "out_peak"),
+                                    _dev(out_dur, torch.int64, "out_dur"),
+                                    _dev(out_feasible, torch.int32, "out_feasible"), _stream())
+    _check(rc, "moc_eval_batch_noalloc")
     return out_peak, out_dur, out_feasible
 
 

@@ -448,6 +448,77 @@ int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps
     return MOC_OK;
 }
 
+// ---- evaluation without any allocation -----------------------------------------------------------
+// Packing offsets for moc_eval_batch_noalloc live in this array of the library's device image.  In
+// host code `g_noalloc_offs` is only a stand-in for the symbol, not a device address: the address a
+// kernel can use comes from cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) long long g_noalloc_offs[MOC_NOALLOC_MAX_B + 1];
+
+namespace {
+constexpr int kMaxDevices = 64;
+int64_t* g_noalloc_ptr[kMaxDevices] = {};  // device address of g_noalloc_offs, per device ordinal
+
+// Caller has made `device` current.
+int noalloc_offsets(int device, int64_t** out) {
+    if (device < 0 || device >= kMaxDevices) return fail(MOC_ERR_ARG, "device ordinal %d not supported", device);
+    int64_t* ptr = __atomic_load_n(&g_noalloc_ptr[device], __ATOMIC_ACQUIRE);
+    if (!ptr) {
+        cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_offs);
+        if (e != cudaSuccess || !ptr)
+            return fail(MOC_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e));
+        __atomic_store_n(&g_noalloc_ptr[device], ptr, __ATOMIC_RELEASE);
+    }
+    *out = ptr;
+    return MOC_OK;
+}
+}  // namespace
+
+int moc_eval_batch_noalloc(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B,
+                           int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
+                           void* stream) {
+    g_err[0] = 0;
+    g_launches = 0;
+    if (!g || B < 0) return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: null handle or B < 0");
+    if (B == 0) return MOC_OK;
+    if (B > MOC_NOALLOC_MAX_B)
+        return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: B = %d exceeds the fixed scratch of %d sequences; "
+                    "split the batch or use moc_eval_batch", B, MOC_NOALLOC_MAX_B);
+    if (!seqs || !lens || !out_peak || !out_dur || !out_feasible)
+        return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: null array");
+    if (reinterpret_cast<uintptr_t>(seqs) & 3) return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: seqs not 4-byte aligned");
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    int64_t* offs = nullptr;
+    int rc = noalloc_offsets(g->device, &offs);
+    if (rc != MOC_OK) return rc;
+    if (!g->plan_eval.valid) {
+        rc = make_plan(g, false, &g->plan_eval);  // attribute and occupancy queries only
+        if (rc != MOC_OK) return rc;
+    }
+    const Plan& pl = g->plan_eval;
+    if (pl.global_state)
+        return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: this graph needs a global workspace "
+                    "(per-sequence state exceeds shared memory); use moc_eval_batch");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, offs);  // rewrites offs[0..B] before any use
+    ++g_launches;
+    moc::EvalParams p = base_params(g, pl);
+    p.seqs = seqs;
+    p.lens = lens;
+    p.offs = offs;
+    p.B = B;
+    p.M = M;
+    p.out_peak = out_peak;
+    p.out_dur = out_dur;
+    p.out_status = out_feasible;
+    p.gstate = nullptr;
+    pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
+    ++g_launches;
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+
 int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t* out_profile,
                     int32_t* out_free, int32_t* out_status, void* stream) {
     g_err[0] = 0;
