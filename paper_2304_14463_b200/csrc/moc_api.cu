@@ -9,6 +9,7 @@
 
 #include "../../include/moc.h"
 #include "moc_kernels.cuh"
+#include "moc_pair_kernel.cuh"
 
 namespace {
 
@@ -32,6 +33,7 @@ int fail(int code, const char* fmt, ...) {
     } while (0)
 
 using KernelFn = void (*)(const moc::EvalParams);
+using PairFn = void (*)(const moc::PairParams);
 
 struct Plan {
     bool valid = false;
@@ -40,6 +42,10 @@ struct Plan {
     size_t smem = 0;
     bool global_state = false, wide = false;
     uint32_t cnt_bytes = 0, occ_bytes = 0, delta_bytes = 0, group_bytes = 0;
+    // fast path for C <= 2: a warp per sequence, graph staged in shared memory
+    bool pair = false;
+    PairFn pair_fn = nullptr;
+    uint32_t nd_bytes = 0, mm_bytes = 0, col_bytes = 0, jds_bytes = 0, word_bytes = 0, list_bytes = 0;
 };
 
 }  // namespace
@@ -58,6 +64,13 @@ struct moc_graph {
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;
     int32_t want_G = 0, want_gpc = 0;
+    // jagged-diagonal successor lists in out-degree order (null when n > 32767)
+    int32_t max_deg = 0;
+    uint32_t* d_nd = nullptr;
+    uint16_t* d_jds = nullptr;
+    uint32_t* d_colstart = nullptr;
+    int32_t* d_mm32 = nullptr;
+    int64_t* d_mm64 = nullptr;
     // grow-only scratch; mutable because evaluation takes a const handle
     mutable Plan plan_eval, plan_profile;
     mutable int64_t* d_offs = nullptr;
@@ -124,6 +137,46 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
                  sh_delta = align16((t_max + 1) * mem_sz);
     const size_t sh_group = sh_cnt + sh_occ + sh_delta + align16(moc::kRedBytes);
     const size_t smem_cap = g->smem_optin > 1024 ? g->smem_optin - 1024 : 0;  // 1 KB per block is reserved
+    if (!profile && g->want_G == 0 && C <= 2 && g->d_nd != nullptr) {
+        // warp-per-sequence fast path
+        const size_t msz = pl.wide ? 8 : 4, per_vec = 16 / msz;
+        const size_t nvec_d = (t_max + 1 + per_vec - 1) / per_vec;
+        const size_t v_max = ((nvec_d + 31) / 32) | 1;
+        const size_t nd_b = align16(4 * n), mm_b = align16(msz * n), col_b = align16(4 * ((size_t)g->max_deg + 1)),
+                     jds_b = align16(2 * (size_t)g->n_edges), word_b = align16(4 * n),
+                     delta_b = moc::kPairDeltaFront + 32 * v_max * 16, list_b = align16(2 * n);
+        const size_t graph_b = nd_b + mm_b + col_b + jds_b, warp_b = word_b + delta_b + list_b;
+        PairFn fn = pl.wide ? (PairFn)moc::eval_pair_kernel<int64_t> : (PairFn)moc::eval_pair_kernel<int32_t>;
+        int best_wpb = 0, best_warps = 0, best_nb = 0;
+        const int cand[4] = {16, 12, 8, 4};
+        for (int ci = 0; ci < 4; ++ci) {
+            const int wpb = g->want_gpc ? std::min(g->want_gpc, 16) : cand[ci];
+            const size_t sm = graph_b + wpb * warp_b;
+            if (sm > smem_cap) { if (g->want_gpc) break; else continue; }
+            if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) { cudaGetLastError(); continue; }
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, wpb * 32, sm) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (nb * wpb > best_warps) { best_warps = nb * wpb; best_wpb = wpb; best_nb = nb; }
+            if (g->want_gpc) break;
+        }
+        if (best_warps >= 8) {
+            pl.pair = true;
+            pl.pair_fn = fn;
+            pl.G = 32;
+            pl.gpc = best_wpb;
+            pl.block = 32 * best_wpb;
+            pl.smem = graph_b + best_wpb * warp_b;
+            pl.grid = g->sm_count * best_nb;
+            pl.nd_bytes = (uint32_t)nd_b; pl.mm_bytes = (uint32_t)mm_b; pl.col_bytes = (uint32_t)col_b;
+            pl.jds_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
+            pl.list_bytes = (uint32_t)list_b;
+            cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+            if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            pl.valid = true;
+            *out = pl;
+            return MOC_OK;
+        }
+    }
     if (t_max <= 65534 && sh_group <= smem_cap) {
         pl.global_state = false;
         pl.cnt_bytes = (uint32_t)sh_cnt;
@@ -220,6 +273,54 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     return p;
 }
 
+// Enqueues the offsets kernel and the evaluation kernel of plan `pl` with `offs` as scratch.
+int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_t* seqs, const int32_t* lens,
+                 int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
+                 cudaStream_t st) {
+    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, offs);
+    ++g_launches;
+    if (pl.pair) {
+        moc::PairParams q{};
+        q.n = g->n;
+        q.n_edges = (int32_t)g->n_edges;
+        q.max_deg = g->max_deg;
+        q.max_T = g->C * g->n;
+        q.nd = g->d_nd;
+        q.jds = g->d_jds;
+        q.colstart = g->d_colstart;
+        q.mm = pl.wide ? (const void*)g->d_mm64 : (const void*)g->d_mm32;
+        q.w = g->d_w;
+        q.base_dur = g->sum_w;
+        q.seqs = seqs;
+        q.lens = lens;
+        q.offs = offs;
+        q.B = B;
+        q.M = M;
+        q.out_peak = out_peak;
+        q.out_dur = out_dur;
+        q.out_status = out_feasible;
+        q.nd_bytes = pl.nd_bytes; q.mm_bytes = pl.mm_bytes; q.col_bytes = pl.col_bytes; q.jds_bytes = pl.jds_bytes;
+        q.word_bytes = pl.word_bytes; q.delta_bytes = pl.delta_bytes; q.list_bytes = pl.list_bytes;
+        pl.pair_fn<<<grid, pl.block, pl.smem, st>>>(q);
+    } else {
+        moc::EvalParams p = base_params(g, pl);
+        p.seqs = seqs;
+        p.lens = lens;
+        p.offs = offs;
+        p.B = B;
+        p.M = M;
+        p.out_peak = out_peak;
+        p.out_dur = out_dur;
+        p.out_status = out_feasible;
+        p.gstate = g->d_state;
+        pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
+    }
+    ++g_launches;
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+
 int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B, int64_t M,
                 int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st) {
     if (!g->plan_eval.valid) {
@@ -229,27 +330,11 @@ int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, in
     const Plan& pl = g->plan_eval;
     int rc = ensure((void**)&g->d_offs, &g->offs_cap, ((size_t)B + 1) * sizeof(int64_t));
     if (rc != MOC_OK) return rc;
-    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
     if (pl.global_state) {
         rc = ensure((void**)&g->d_state, &g->state_cap, (size_t)pl.grid * pl.group_bytes);
         if (rc != MOC_OK) return rc;
     }
-    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, g->d_offs);
-    ++g_launches;
-    moc::EvalParams p = base_params(g, pl);
-    p.seqs = seqs;
-    p.lens = lens;
-    p.offs = g->d_offs;
-    p.B = B;
-    p.M = M;
-    p.out_peak = out_peak;
-    p.out_dur = out_dur;
-    p.out_status = out_feasible;
-    p.gstate = g->d_state;
-    pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
-    ++g_launches;
-    MOC_CUDA(cudaGetLastError());
-    return MOC_OK;
+    return enqueue_eval(g, pl, g->d_offs, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
 }
 
 }  // namespace
@@ -342,6 +427,42 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     up((void**)&g->d_w, w, (size_t)n * 8);
     up((void**)&g->d_m64, m, (size_t)n * 8);
     up((void**)&g->d_m32, m32.data(), (size_t)n * 4);
+    if (n <= 32767) {
+        // successor lists in jagged-diagonal form: nodes sorted by out-degree (descending, ties by
+        // id); column k lists the k-th successor of every node whose out-degree exceeds k
+        try {
+            std::vector<int32_t> order((size_t)n);
+            for (int32_t v = 0; v < n; ++v) order[v] = v;
+            auto deg = [&](int32_t v) { return succ_start[v + 1] - succ_start[v]; };
+            std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
+            const int32_t max_deg = deg(order[0]);
+            std::vector<uint32_t> nd((size_t)n), colstart((size_t)max_deg + 1, 0);
+            std::vector<uint16_t> jds((size_t)std::max<int64_t>(ne, 1));
+            std::vector<int32_t> mm32((size_t)n);
+            std::vector<int64_t> mm64((size_t)n);
+            for (int32_t i = 0; i < n; ++i) {
+                nd[i] = (uint32_t)order[i] | ((uint32_t)deg(order[i]) << 16);
+                mm32[i] = m32[order[i]];
+                mm64[i] = m[order[i]];
+            }
+            uint32_t pos = 0;
+            for (int32_t k = 0; k < max_deg; ++k) {
+                colstart[k] = pos;
+                for (int32_t i = 0; i < n && deg(order[i]) > k; ++i)
+                    jds[pos++] = (uint16_t)succ[succ_start[order[i]] + k];
+            }
+            colstart[max_deg] = pos;
+            g->max_deg = max_deg;
+            up((void**)&g->d_nd, nd.data(), (size_t)n * 4);
+            up((void**)&g->d_jds, jds.data(), (size_t)ne * 2);
+            up((void**)&g->d_colstart, colstart.data(), ((size_t)max_deg + 1) * 4);
+            up((void**)&g->d_mm32, mm32.data(), (size_t)n * 4);
+            up((void**)&g->d_mm64, mm64.data(), (size_t)n * 8);
+        } catch (const std::bad_alloc&) {
+            moc_graph_destroy(g);
+            return fail(MOC_ERR_NOMEM, "host allocation failed");
+        }
+    }
     if (e != cudaSuccess) {
         rc = fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA,
                   "moc_graph_create: %s", cudaGetErrorString(e));
@@ -381,6 +502,11 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_w);
     cudaFree(g->d_m64);
     cudaFree(g->d_m32);
+    cudaFree(g->d_nd);
+    cudaFree(g->d_jds);
+    cudaFree(g->d_colstart);
+    cudaFree(g->d_mm32);
+    cudaFree(g->d_mm64);
     cudaFree(g->d_offs);
     cudaFree(g->d_state);
     cudaFree(g->d_stage_seqs);
@@ -499,24 +625,8 @@ int moc_eval_batch_noalloc(const moc_graph* g, const int32_t* seqs, const int32_
     if (pl.global_state)
         return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: this graph needs a global workspace "
                     "(per-sequence state exceeds shared memory); use moc_eval_batch");
-    cudaStream_t st = (cudaStream_t)stream;
-    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
-    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, offs);  // rewrites offs[0..B] before any use
-    ++g_launches;
-    moc::EvalParams p = base_params(g, pl);
-    p.seqs = seqs;
-    p.lens = lens;
-    p.offs = offs;
-    p.B = B;
-    p.M = M;
-    p.out_peak = out_peak;
-    p.out_dur = out_dur;
-    p.out_status = out_feasible;
-    p.gstate = nullptr;
-    pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
-    ++g_launches;
-    MOC_CUDA(cudaGetLastError());
-    return MOC_OK;
+    // the offsets kernel rewrites offs[0..B] before the evaluation kernel reads them
+    return enqueue_eval(g, pl, offs, seqs, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream);
 }
 
 int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t* out_profile,

@@ -124,7 +124,7 @@ def test_mem_profile_parity(B, idx):
 
 
 # ------------------------------------------------------------------ launch shapes, alignment, edges
-@pytest.mark.parametrize("tps,spb", [(32, 1), (32, 8), (32, 16), (64, 4), (128, 2), (256, 1), (256, 3),
+@pytest.mark.parametrize("tps,spb", [(0, 0), (0, 4), (0, 8), (0, 12), (0, 16), (32, 1), (32, 8), (32, 16), (64, 4), (128, 2), (256, 1), (256, 3),
                                      (512, 1), (512, 2), (1024, 1)])
 def test_every_launch_shape(B, tps, spb):
     wl = W.make(2, seed=6, B=700)
