@@ -10,7 +10,8 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmoc_b200.so")
+# MOC_B200_LIB selects another build of the same library (e.g. one compiled with other flags)
+LIB_PATH = os.environ.get("MOC_B200_LIB") or os.path.join(_HERE, "libmoc_b200.so")
 
 MOC_OK = 0
 ERROR_NAMES = {-1: "MOC_ERR_ARG", -2: "MOC_ERR_RANGE", -3: "MOC_ERR_CYCLE", -4: "MOC_ERR_OVERFLOW",

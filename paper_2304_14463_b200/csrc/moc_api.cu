@@ -45,7 +45,7 @@ struct Plan {
     // fast path for C <= 2: a warp per sequence, graph staged in shared memory
     bool pair = false;
     PairFn pair_fn = nullptr;
-    uint32_t nd_bytes = 0, mm_bytes = 0, col_bytes = 0, jds_bytes = 0, word_bytes = 0, list_bytes = 0;
+    uint32_t rec_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
 };
 
 }  // namespace
@@ -64,13 +64,12 @@ struct moc_graph {
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;
     int32_t want_G = 0, want_gpc = 0;
-    // jagged-diagonal successor lists in out-degree order (null when n > 32767)
-    int32_t max_deg = 0;
-    uint32_t* d_nd = nullptr;
-    uint16_t* d_jds = nullptr;
-    uint32_t* d_colstart = nullptr;
-    int32_t* d_mm32 = nullptr;
-    int64_t* d_mm64 = nullptr;
+    // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
+    int32_t sell_len = 0, n_slices = 0;
+    void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
+    void* d_rec64 = nullptr;
+    uint16_t* d_sell = nullptr;
+    uint32_t* d_tile = nullptr;
     // grow-only scratch; mutable because evaluation takes a const handle
     mutable Plan plan_eval, plan_profile;
     mutable int64_t* d_offs = nullptr;
@@ -137,15 +136,15 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
                  sh_delta = align16((t_max + 1) * mem_sz);
     const size_t sh_group = sh_cnt + sh_occ + sh_delta + align16(moc::kRedBytes);
     const size_t smem_cap = g->smem_optin > 1024 ? g->smem_optin - 1024 : 0;  // 1 KB per block is reserved
-    if (!profile && g->want_G == 0 && C <= 2 && g->d_nd != nullptr) {
+    if (!profile && g->want_G == 0 && C <= 2 && g->d_rec32 != nullptr) {
         // warp-per-sequence fast path
         const size_t msz = pl.wide ? 8 : 4, per_vec = 16 / msz;
         const size_t nvec_d = (t_max + 1 + per_vec - 1) / per_vec;
         const size_t v_max = ((nvec_d + 31) / 32) | 1;
-        const size_t nd_b = align16(4 * n), mm_b = align16(msz * n), col_b = align16(4 * ((size_t)g->max_deg + 1)),
-                     jds_b = align16(2 * (size_t)g->n_edges), word_b = align16(4 * n),
-                     delta_b = moc::kPairDeltaFront + 32 * v_max * 16, list_b = align16(2 * n);
-        const size_t graph_b = nd_b + mm_b + col_b + jds_b, warp_b = word_b + delta_b + list_b;
+        const size_t rec_b = align16((pl.wide ? sizeof(moc::NodeRec<int64_t>) : sizeof(moc::NodeRec<int32_t>)) * n),
+                     col_b = align16(4 * (size_t)g->n_slices), jds_b = align16(2 * (size_t)g->sell_len),
+                     word_b = align16(4 * (n + 1)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
+        const size_t graph_b = rec_b + col_b + jds_b, warp_b = word_b + delta_b;
         PairFn fn = pl.wide ? (PairFn)moc::eval_pair_kernel<int64_t> : (PairFn)moc::eval_pair_kernel<int32_t>;
         int best_wpb = 0, best_warps = 0, best_nb = 0;
         const int cand[4] = {16, 12, 8, 4};
@@ -167,9 +166,8 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             pl.block = 32 * best_wpb;
             pl.smem = graph_b + best_wpb * warp_b;
             pl.grid = g->sm_count * best_nb;
-            pl.nd_bytes = (uint32_t)nd_b; pl.mm_bytes = (uint32_t)mm_b; pl.col_bytes = (uint32_t)col_b;
-            pl.jds_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
-            pl.list_bytes = (uint32_t)list_b;
+            pl.rec_bytes = (uint32_t)rec_b; pl.tile_bytes = (uint32_t)col_b;
+            pl.sell_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
             cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
             if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
             pl.valid = true;
@@ -278,18 +276,29 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
                  int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
                  cudaStream_t st) {
     const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
-    moc::offsets_kernel<<<1, 1024, 0, st>>>(lens, B, offs);
+    moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
     ++g_launches;
+    // the evaluation kernel may begin (stage the graph, set up shared memory) while the offsets
+    // kernel still runs; it waits for the offsets inside
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)pl.block);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (pl.pair) {
         moc::PairParams q{};
         q.n = g->n;
-        q.n_edges = (int32_t)g->n_edges;
-        q.max_deg = g->max_deg;
+        q.sell_len = g->sell_len;
+        q.n_slices = g->n_slices;
         q.max_T = g->C * g->n;
-        q.nd = g->d_nd;
-        q.jds = g->d_jds;
-        q.colstart = g->d_colstart;
-        q.mm = pl.wide ? (const void*)g->d_mm64 : (const void*)g->d_mm32;
+        q.rec = pl.wide ? g->d_rec64 : g->d_rec32;
+        q.sell = g->d_sell;
+        q.tile = g->d_tile;
         q.w = g->d_w;
         q.base_dur = g->sum_w;
         q.seqs = seqs;
@@ -300,9 +309,9 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
         q.out_peak = out_peak;
         q.out_dur = out_dur;
         q.out_status = out_feasible;
-        q.nd_bytes = pl.nd_bytes; q.mm_bytes = pl.mm_bytes; q.col_bytes = pl.col_bytes; q.jds_bytes = pl.jds_bytes;
-        q.word_bytes = pl.word_bytes; q.delta_bytes = pl.delta_bytes; q.list_bytes = pl.list_bytes;
-        pl.pair_fn<<<grid, pl.block, pl.smem, st>>>(q);
+        q.rec_bytes = pl.rec_bytes; q.tile_bytes = pl.tile_bytes; q.sell_bytes = pl.sell_bytes;
+        q.word_bytes = pl.word_bytes; q.delta_bytes = pl.delta_bytes;
+        MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.pair_fn, q));
     } else {
         moc::EvalParams p = base_params(g, pl);
         p.seqs = seqs;
@@ -314,7 +323,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
         p.out_dur = out_dur;
         p.out_status = out_feasible;
         p.gstate = g->d_state;
-        pl.fn<<<grid, pl.block, pl.smem, st>>>(p);
+        MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.fn, p));
     }
     ++g_launches;
     MOC_CUDA(cudaGetLastError());
@@ -427,37 +436,50 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     up((void**)&g->d_w, w, (size_t)n * 8);
     up((void**)&g->d_m64, m, (size_t)n * 8);
     up((void**)&g->d_m32, m32.data(), (size_t)n * 4);
-    if (n <= 32767) {
-        // successor lists in jagged-diagonal form: nodes sorted by out-degree (descending, ties by
-        // id); column k lists the k-th successor of every node whose out-degree exceeds k
+    if (n <= 16383) {
+        // successor lists as a sliced ELL matrix: nodes sorted by out-degree (descending, ties by
+        // id) in slices of 32; slice s is a [degree of its first node][32] tile of byte offsets
+        // 4*successor, padded with 4*n (a dummy word).  Skipped when padding would more than
+        // double the storage (a few very high degrees): such graphs use the general kernel.
         try {
             std::vector<int32_t> order((size_t)n);
             for (int32_t v = 0; v < n; ++v) order[v] = v;
             auto deg = [&](int32_t v) { return succ_start[v + 1] - succ_start[v]; };
             std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
-            const int32_t max_deg = deg(order[0]);
-            std::vector<uint32_t> nd((size_t)n), colstart((size_t)max_deg + 1, 0);
-            std::vector<uint16_t> jds((size_t)std::max<int64_t>(ne, 1));
-            std::vector<int32_t> mm32((size_t)n);
-            std::vector<int64_t> mm64((size_t)n);
-            for (int32_t i = 0; i < n; ++i) {
-                nd[i] = (uint32_t)order[i] | ((uint32_t)deg(order[i]) << 16);
-                mm32[i] = m32[order[i]];
-                mm64[i] = m[order[i]];
+            const int32_t n_slices = (n + 31) / 32;
+            int64_t sell_len = 0;
+            for (int32_t s = 0; s < n_slices; ++s) sell_len += 32 * (int64_t)deg(order[32 * s]);
+            if (sell_len <= 2 * ne + 32 * 64 && sell_len < (1 << 18)) {
+                std::vector<uint32_t> tile((size_t)n_slices);
+                std::vector<moc::NodeRec<int32_t>> rec32((size_t)n);
+                std::vector<moc::NodeRec<int64_t>> rec64((size_t)n);
+                std::vector<uint16_t> sell((size_t)std::max<int64_t>(sell_len, 1), (uint16_t)(4 * n));
+                for (int32_t i = 0; i < n; ++i) {
+                    const uint32_t nd = 4u * (uint32_t)order[i] | ((uint32_t)deg(order[i]) << 16);
+                    rec32[i].nd = nd;
+                    rec32[i].m = m32[order[i]];
+                    rec64[i].nd = nd;
+                    rec64[i].pad = 0;
+                    rec64[i].m = m[order[i]];
+                }
+                uint32_t pos = 0;
+                for (int32_t s = 0; s < n_slices; ++s) {
+                    const int32_t rows = deg(order[32 * s]);
+                    tile[s] = pos | ((uint32_t)rows << 18);
+                    for (int32_t l = 0; l < 32 && 32 * s + l < n; ++l) {
+                        const int32_t u = order[32 * s + l];
+                        for (int32_t k = 0; k < deg(u); ++k)
+                            sell[pos + 32 * k + l] = (uint16_t)(4 * succ[succ_start[u] + k]);
+                    }
+                    pos += 32 * (uint32_t)rows;
+                }
+                g->sell_len = (int32_t)sell_len;
+                g->n_slices = n_slices;
+                up(&g->d_rec32, rec32.data(), (size_t)n * sizeof(rec32[0]));
+                up(&g->d_rec64, rec64.data(), (size_t)n * sizeof(rec64[0]));
+                up((void**)&g->d_sell, sell.data(), (size_t)sell_len * 2);
+                up((void**)&g->d_tile, tile.data(), (size_t)n_slices * 4);
             }
-            uint32_t pos = 0;
-            for (int32_t k = 0; k < max_deg; ++k) {
-                colstart[k] = pos;
-                for (int32_t i = 0; i < n && deg(order[i]) > k; ++i)
-                    jds[pos++] = (uint16_t)succ[succ_start[order[i]] + k];
-            }
-            colstart[max_deg] = pos;
-            g->max_deg = max_deg;
-            up((void**)&g->d_nd, nd.data(), (size_t)n * 4);
-            up((void**)&g->d_jds, jds.data(), (size_t)ne * 2);
-            up((void**)&g->d_colstart, colstart.data(), ((size_t)max_deg + 1) * 4);
-            up((void**)&g->d_mm32, mm32.data(), (size_t)n * 4);
-            up((void**)&g->d_mm64, mm64.data(), (size_t)n * 8);
         } catch (const std::bad_alloc&) {
             moc_graph_destroy(g);
             return fail(MOC_ERR_NOMEM, "host allocation failed");
@@ -502,11 +524,10 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_w);
     cudaFree(g->d_m64);
     cudaFree(g->d_m32);
-    cudaFree(g->d_nd);
-    cudaFree(g->d_jds);
-    cudaFree(g->d_colstart);
-    cudaFree(g->d_mm32);
-    cudaFree(g->d_mm64);
+    cudaFree(g->d_rec32);
+    cudaFree(g->d_rec64);
+    cudaFree(g->d_sell);
+    cudaFree(g->d_tile);
     cudaFree(g->d_offs);
     cudaFree(g->d_state);
     cudaFree(g->d_stage_seqs);

@@ -54,6 +54,14 @@ template <typename PosT> struct PosNone;
 template <> struct PosNone<uint16_t> { static constexpr uint32_t value = 0xFFFFu; };
 template <> struct PosNone<int32_t> { static constexpr uint32_t value = 0x7FFFFFFFu; };
 
+// Waits until the kernel launched before this one in the stream has finished and its writes are
+// visible (no-op unless this kernel was launched with programmatic stream serialization).
+__device__ __forceinline__ void wait_for_previous_kernel() {
+#if __CUDA_ARCH__ >= 900
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+
 template <int G>
 __device__ __forceinline__ void group_sync(int bar_id) {
     if constexpr (G == 32) {
@@ -322,6 +330,7 @@ __device__ __forceinline__ void eval_one(const EvalParams& p, const int b, const
 template <int G, typename MemT, int CP, bool kProfile>
 __global__ void __launch_bounds__(1024) eval_shared_kernel(const EvalParams p) {
     extern __shared__ __align__(16) char smem[];
+    wait_for_previous_kernel();
     const int gpc = blockDim.x / G;
     const int gi = threadIdx.x / G, tid = threadIdx.x % G;
     char* state = smem + (size_t)gi * p.group_bytes;
@@ -335,48 +344,61 @@ __global__ void __launch_bounds__(1024) eval_shared_kernel(const EvalParams p) {
 template <int CP, bool kProfile>
 __global__ void __launch_bounds__(1024) eval_global_kernel(const EvalParams p) {
     char* state = p.gstate + (size_t)blockIdx.x * p.group_bytes;
+    wait_for_previous_kernel();
     for (int b = blockIdx.x; b < p.B; b += gridDim.x)
         eval_one<1024, int64_t, int32_t, CP, kProfile>(p, b, threadIdx.x, 0, state);
 }
 
-// offs = exclusive prefix sum of max(lens, 0); offs[B] = total.  One block.
-__global__ void __launch_bounds__(1024) offsets_kernel(const int32_t* __restrict__ lens, int32_t B,
-                                                       int64_t* __restrict__ offs) {
-    constexpr int kPer = 8, kTile = 1024 * kPer;
-    __shared__ int32_t tile[kTile];
-    __shared__ int64_t wsum[32];
-    __shared__ int64_t carry_s;
+// offs = exclusive prefix sum of max(lens, 0); offs[B] = total.
+// Block j owns elements [j*kOffsTile, (j+1)*kOffsTile): it first adds up everything in front of its
+// tile (redundantly with the other blocks -- B is small, and this needs no cross-block handshake),
+// then scans its own tile.  The dependent evaluation kernel may start its prologue at once.
+constexpr int kOffsThreads = 512;
+constexpr int kOffsPer = 4;
+constexpr int kOffsTile = kOffsThreads * kOffsPer;
+
+__global__ void __launch_bounds__(kOffsThreads) offsets_kernel(const int32_t* __restrict__ lens, int32_t B,
+                                                                int64_t* __restrict__ offs) {
+#if __CUDA_ARCH__ >= 900
+    asm volatile("griddepcontrol.launch_dependents;");
+#endif
+    __shared__ int64_t wsum[kOffsThreads / 32];
+    __shared__ int64_t wtot[kOffsThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) carry_s = 0;
-    __syncthreads();
-    for (int64_t base = 0; base < B; base += kTile) {
-        for (int k = 0; k < kPer; ++k) {
-            const int64_t i = base + k * 1024 + tid;
-            int32_t v = i < B ? lens[i] : 0;
-            tile[k * 1024 + tid] = v > 0 ? v : 0;
-        }
-        __syncthreads();
-        int64_t s = 0;
-        int32_t loc[kPer];
-#pragma unroll
-        for (int k = 0; k < kPer; ++k) { loc[k] = tile[tid * kPer + k]; s += loc[k]; }
-        int64_t incl = warp_inclusive_sum(s, lane);
-        if (lane == 31) wsum[warp] = incl;
-        __syncthreads();
-        int64_t prefix = carry_s;
-        for (int k = 0; k < warp; ++k) prefix += wsum[k];
-        int64_t run = prefix + incl - s;
-#pragma unroll
-        for (int k = 0; k < kPer; ++k) {
-            const int64_t i = base + tid * kPer + k;
-            if (i < B) offs[i] = run;
-            run += loc[k];
-        }
-        __syncthreads();
-        if (tid == 1023) carry_s = run;
-        __syncthreads();
+    const int64_t tile0 = (int64_t)blockIdx.x * kOffsTile;
+    // ---- sum of everything before the tile
+    int64_t s = 0;
+    for (int64_t i = tid; i < tile0; i += kOffsThreads) {
+        const int32_t v = __ldg(lens + i);
+        s += v > 0 ? v : 0;
     }
-    if (tid == 0) offs[B] = carry_s;
+    s = warp_sum(s);
+    if (lane == 0) wtot[warp] = s;
+    // ---- own tile: kOffsPer consecutive elements per thread
+    int32_t loc[kOffsPer];
+    int64_t t = 0;
+#pragma unroll
+    for (int k = 0; k < kOffsPer; ++k) {
+        const int64_t i = tile0 + tid * kOffsPer + k;
+        const int32_t v = i < B ? __ldg(lens + i) : 0;
+        loc[k] = v > 0 ? v : 0;
+        t += loc[k];
+    }
+    const int64_t incl = warp_inclusive_sum(t, lane);
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    int64_t run = incl - t;
+    for (int k = 0; k < kOffsThreads / 32; ++k) {
+        run += wtot[k];
+        if (k < warp) run += wsum[k];
+    }
+#pragma unroll
+    for (int k = 0; k < kOffsPer; ++k) {
+        const int64_t i = tile0 + tid * kOffsPer + k;
+        if (i < B) offs[i] = run;
+        run += loc[k];
+        if (i == B - 1) offs[B] = run;
+    }
 }
 
 }  // namespace moc

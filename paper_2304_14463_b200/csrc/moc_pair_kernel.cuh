@@ -4,21 +4,27 @@
 //
 // Representation.  Positions are 1-based and 16 bits wide; 0 means "no copy".  Each node owns one
 // 32-bit word holding its (at most two) positions, so a consumer reads both copies of a
-// predecessor/successor with one load.  The successor lists are stored in jagged-diagonal form:
-// nodes are sorted by out-degree (descending) and column k holds the k-th successor of every node
-// that has one, so that lanes working on consecutive sorted nodes read consecutive entries and a
-// warp's trip count is the out-degree of its first lane.
+// predecessor/successor with one load.  The successor lists are stored as a sliced ELL matrix:
+// nodes are sorted by out-degree (descending) and cut into slices of 32; slice s is a dense
+// [degree of its first node][32] tile whose row k holds the k-th successor of each of its nodes, as
+// the byte offset of that successor's word, padded with the offset of a dummy word that stays zero.
+// Lanes read consecutive entries, every lane of a warp runs the same trip count, and the padding
+// is neutral for the maxima and minima taken over the successors.
 //
 // Stages for one sequence seq[0..T) (paper: Section 2, Eqs. 1-8):
 //   1. occurrence words   step t exchanges t+1 into the low half of its node's word and moves the
 //                         previous occupant to the high half.  A third copy loses a position, which
 //                         the check "sum of stored positions == T(T+1)/2" detects; an absent node
 //                         (Eq. 7) shows as a zero low half.
-//   2. free steps         last copy b of u: free = max(b, latest copy of any successor) -- every
-//                         successor copy after b falls in b's window; first copy a of a node
-//                         computed twice: free = latest successor copy inside (a, b), else a
-//                         (Eqs. 2, 3, 5).  A sink's last copy is kept to the end.  Precedence
-//                         (Eq. 5) holds iff no successor copy precedes the first copy of u.
+//   2. free steps         one lane per node u with copies a <= b (a = b if computed once), one pass
+//                         over its successors' words r with three packed 16-bit reductions:
+//                           F = max r            latest successor copy: b is kept until max(b, F);
+//                           D = min (r - 1)      earliest successor copy: before a = Eq. 5 violated;
+//                           G = max (r - b)      mod 2^16 this ranks the copies below b above all
+//                                                others, in order: the latest successor copy inside
+//                                                (a, b), until which the first copy a is kept
+//                                                (Eqs. 2, 3, 5).
+//                         A sink's last copy is kept to the end.
 //   3. memory profile     delta[p] += m_u, delta[free+1] -= m_u, prefix sum (Eq. 4).
 //   4. reductions         peak (Section 2), duration = sum_v w_v + sum over second copies (Eq. 1).
 #pragma once
@@ -31,13 +37,12 @@ namespace moc {
 
 struct PairParams {
     int32_t n;
-    int32_t n_edges;
-    int32_t max_deg;
+    int32_t sell_len;          // entries of the sliced ELL matrix
+    int32_t n_slices;          // ceil(n / 32)
     int32_t max_T;             // C * n
-    const uint32_t* nd;        // n: node id | out-degree << 16, sorted by out-degree descending
-    const uint16_t* jds;       // n_edges successor ids, column after column
-    const uint32_t* colstart;  // max_deg + 1 column starts
-    const void* mm;            // n output sizes (MemT) in sorted-node order
+    const void* rec;           // n node records (NodeRec<MemT>) in out-degree order
+    const uint16_t* sell;      // sell_len byte offsets (4 * successor id, 4 * n = dummy)
+    const uint32_t* tile;      // n_slices: first entry of the slice | rows of the slice << 18
     const int64_t* w;          // n durations by node id
     int64_t base_dur;          // sum of all w
     const int32_t* seqs;
@@ -49,8 +54,8 @@ struct PairParams {
     int64_t* out_dur;
     int32_t* out_status;
     // shared-memory layout, bytes (multiples of 16)
-    uint32_t nd_bytes, mm_bytes, col_bytes, jds_bytes;  // graph, once per block
-    uint32_t word_bytes, delta_bytes, list_bytes;       // per warp
+    uint32_t rec_bytes, tile_bytes, sell_bytes;  // graph, once per block
+    uint32_t word_bytes, delta_bytes;                  // per warp
 };
 
 constexpr int kPairDeltaFront = 16;  // bytes in front of delta[0]: lands writes of absent nodes
@@ -60,42 +65,61 @@ __device__ __forceinline__ int64_t warp_sum64(int64_t v) {
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
     return v;
 }
+// per-halfword unsigned max / min of two packed 16-bit pairs (one instruction on sm_90 and later)
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t add_u16x2(uint32_t a, uint32_t b) {  // per halfword, wraps
+    uint32_t d;
+    asm("add.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Node record: byte offset of the node's word (4 * id) | out-degree << 16, and its output size.
+template <typename MemT> struct NodeRec;
+template <> struct __align__(8) NodeRec<int32_t> { uint32_t nd; int32_t m; };
+template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; int64_t m; };
+
 __device__ __forceinline__ int32_t warp_max_t(int32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
 __device__ __forceinline__ int64_t warp_max_t(int64_t v) { return warp_max(v); }
 
 template <typename MemT>
 __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     extern __shared__ __align__(16) char smem[];
+    using Rec = NodeRec<MemT>;
     // ---- graph -> shared memory, once per block
-    uint32_t* s_nd = reinterpret_cast<uint32_t*>(smem);
-    MemT* s_mm = reinterpret_cast<MemT*>(smem + p.nd_bytes);
-    uint32_t* s_col = reinterpret_cast<uint32_t*>(smem + p.nd_bytes + p.mm_bytes);
-    uint16_t* s_jds = reinterpret_cast<uint16_t*>(smem + p.nd_bytes + p.mm_bytes + p.col_bytes);
-    const uint32_t graph_bytes = p.nd_bytes + p.mm_bytes + p.col_bytes + p.jds_bytes;
+    Rec* s_rec = reinterpret_cast<Rec*>(smem);
+    uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem + p.rec_bytes);
+    uint16_t* s_sell = reinterpret_cast<uint16_t*>(smem + p.rec_bytes + p.tile_bytes);
+    const uint32_t graph_bytes = p.rec_bytes + p.tile_bytes + p.sell_bytes;
     {
-        const int n = p.n;
-        const MemT* gm = reinterpret_cast<const MemT*>(p.mm);
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            s_nd[i] = __ldg(&p.nd[i]);
-            s_mm[i] = __ldg(&gm[i]);
-        }
-        for (int i = threadIdx.x; i <= p.max_deg; i += blockDim.x) s_col[i] = __ldg(&p.colstart[i]);
-        for (int i = threadIdx.x; i < p.n_edges; i += blockDim.x) s_jds[i] = __ldg(&p.jds[i]);
+        const Rec* grec = reinterpret_cast<const Rec*>(p.rec);
+        for (int i = threadIdx.x; i < p.n; i += blockDim.x) s_rec[i] = grec[i];
+        for (int i = threadIdx.x; i < p.n_slices; i += blockDim.x) s_tile[i] = __ldg(&p.tile[i]);
+        for (int i = threadIdx.x; i < p.sell_len; i += blockDim.x) s_sell[i] = __ldg(&p.sell[i]);
     }
     __syncthreads();
+    wait_for_previous_kernel();  // the packing offsets come from the kernel launched just before
 
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
-    const uint32_t warp_bytes = p.word_bytes + p.delta_bytes + p.list_bytes;
-    char* ws = smem + graph_bytes + (size_t)warp * warp_bytes;
+    const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    // broadcast from lane 0 so that the compiler knows the warp index is uniform across the warp
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
+    char* ws = smem + graph_bytes + (size_t)warp * (p.word_bytes + p.delta_bytes);
     uint32_t* word = reinterpret_cast<uint32_t*>(ws);
     uint16_t* word16 = reinterpret_cast<uint16_t*>(ws);
     char* delta_base = ws + p.word_bytes;                          // includes the front pad
     MemT* delta = reinterpret_cast<MemT*>(delta_base + kPairDeltaFront);
-    uint16_t* list = reinterpret_cast<uint16_t*>(ws + p.word_bytes + p.delta_bytes);
     const int n = p.n;
     const int n_warps = gridDim.x * wpb;
-    const uint32_t lt_mask = (1u << lane) - 1u;
     constexpr int kPerVec = 16 / (int)sizeof(MemT);  // delta entries per 16-byte vector
+    constexpr int kRegVecs = sizeof(MemT) == 4 ? 7 : 0;  // scan keeps up to this many vectors per lane in registers
 
     for (int b = blockIdx.x * wpb + warp; b < p.B; b += n_warps) {
         const int64_t off = p.offs[b];
@@ -153,70 +177,59 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             }
             __syncwarp();
 
-            // ---- stage 2, last copies: one lane per node in out-degree order
+            // ---- stage 2 and the scatter of stage 3: one lane per node, slices in out-degree order
             uint32_t vmin = 0xFFFFFFFFu, vsum = 0;
             bool dep = false;
-            int n_dbl = 0;
-            for (int i0 = 0; i0 < n; i0 += 32) {
+            int64_t dur_extra = 0;
+            for (int i0 = 0, sl = 0; i0 < n; i0 += 32, ++sl) {
                 const int i = i0 + lane;
-                bool dbl = false;
-                if (i < n) {
-                    const uint32_t nd = s_nd[i];
-                    const uint32_t u = nd & 0xFFFFu, deg = nd >> 16;
-                    const uint32_t own = word[u];
-                    const uint32_t lo = own & 0xFFFFu, hi = own >> 16;
+                const bool live = i < n;
+                Rec rec;
+                rec.nd = 4u * (uint32_t)n;  // lanes past the last node look at the dummy word
+                rec.m = 0;
+                if (live) rec = s_rec[i];
+                const uint32_t own = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(word) + (rec.nd & 0xFFFFu));
+                const uint32_t lo = own & 0xFFFFu, hi = own >> 16;
+                const bool dbl = hi != 0;
+                const uint32_t hh = dbl ? hi : lo;
+                const uint32_t a = min(lo, hh), bpos = max(lo, hh);
+                const uint32_t nbb = ((0x10000u - bpos) & 0xFFFFu) * 0x10001u;   // -b in both halves
+                // successors of the slice: uniform trip count, padded entries read the dummy word
+                const uint32_t tl = __shfl_sync(0xFFFFFFFFu, s_tile[sl], 0);
+                const uint16_t* pj = s_sell + (tl & 0x3FFFFu) + lane;
+                const int rows = (int)(tl >> 18);
+                uint32_t F = 0, D = 0xFFFFFFFFu, G = 0;
+#pragma unroll 4
+                for (int k = 0; k < rows; ++k) {
+                    const uint32_t v4 = pj[k * 32];
+                    const uint32_t r = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(word) + v4);
+                    F = max_u16x2(F, r);
+                    D = min_u16x2(D, r - 0x00010001u);   // empty half -> 0xFFFF
+                    G = max_u16x2(G, add_u16x2(r, nbb));
+                }
+                if (live) {
+                    const uint32_t deg = rec.nd >> 16;
                     vmin = min(vmin, lo);
                     vsum += lo + hi;
-                    dbl = hi != 0;
-                    const uint32_t hh = dbl ? hi : lo;
-                    const uint32_t a = min(lo, hh), bpos = max(lo, hh);
-                    uint32_t F = 0, D = 0xFFFFFFFFu;
-                    for (uint32_t k = 0; k < deg; ++k) {
-                        const uint32_t v = s_jds[s_col[k] + i];
-                        const uint32_t r = word[v];
-                        F = __vmaxu2(F, r);                 // latest copy, per half
-                        D = __vminu2(D, r - 0x00010001u);   // earliest copy (0-based); empty half -> 0xFFFF
-                    }
                     const uint32_t Fm = max(F & 0xFFFFu, F >> 16);
                     const uint32_t Dm = min(D & 0xFFFFu, D >> 16);
                     if (deg != 0 && Dm + 1 < a) dep = true;   // a successor copy before the first copy of u
                     const uint32_t fb = deg != 0 ? max(Fm, bpos) : (uint32_t)T;
-                    const MemT mu = s_mm[i];
-                    atomic_add_mem(&delta[(int)bpos - 1], mu);
-                    atomic_add_mem(&delta[fb], (MemT)(-mu));
+                    atomic_add_mem(&delta[(int)bpos - 1], rec.m);
+                    atomic_add_mem(&delta[fb], (MemT)(-rec.m));
+                    if (dbl) {
+                        // latest successor copy h with a < h < b, if any: (h - b) mod 2^16 is the largest
+                        const uint32_t h = (max(G & 0xFFFFu, G >> 16) + bpos) & 0xFFFFu;
+                        const uint32_t fa = (h - 1u < bpos - 1u) ? h : a;
+                        atomic_add_mem(&delta[(int)a - 1], rec.m);
+                        atomic_add_mem(&delta[fa], (MemT)(-rec.m));
+                        dur_extra += __ldg(&p.w[(rec.nd & 0xFFFFu) >> 2]);
+                    }
                 }
-                const uint32_t mask = __ballot_sync(0xFFFFFFFFu, dbl);
-                if (dbl) list[n_dbl + __popc(mask & lt_mask)] = (uint16_t)i;
-                n_dbl += __popc(mask);
             }
             vmin = __reduce_min_sync(0xFFFFFFFFu, vmin);
             vsum = __reduce_add_sync(0xFFFFFFFFu, vsum);
             const bool well_formed = vmin != 0 && vsum == (uint32_t)T * ((uint32_t)T + 1u) / 2u;
-            __syncwarp();
-
-            // ---- stage 2, first copies of nodes computed twice
-            int64_t dur_extra = 0;
-            if (well_formed) {
-                for (int j = lane; j < n_dbl; j += 32) {
-                    const int i = list[j];
-                    const uint32_t nd = s_nd[i];
-                    const uint32_t u = nd & 0xFFFFu, deg = nd >> 16;
-                    const uint32_t own = word[u];
-                    const uint32_t lo = own & 0xFFFFu, hi = own >> 16;
-                    const uint32_t a = min(lo, hi), bpos = max(lo, hi);
-                    uint32_t fa = a;
-                    for (uint32_t k = 0; k < deg; ++k) {
-                        const uint32_t v = s_jds[s_col[k] + i];
-                        const uint32_t r = word[v];
-                        const uint32_t x = r & 0xFFFFu, y = r >> 16;
-                        fa = max(fa, max(x < bpos ? x : 0u, y < bpos ? y : 0u));
-                    }
-                    const MemT mu = s_mm[i];
-                    atomic_add_mem(&delta[(int)a - 1], mu);
-                    atomic_add_mem(&delta[fa], (MemT)(-mu));
-                    dur_extra += __ldg(&p.w[u]);
-                }
-            }
             dep = __any_sync(0xFFFFFFFFu, dep);
             __syncwarp();
 
@@ -228,28 +241,49 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             } else {
                 // ---- stage 3 + 4: prefix sum and running maximum; lane owns V consecutive vectors
                 const int4* d4 = reinterpret_cast<const int4*>(delta) + lane * V;
-                MemT s = 0;
-                for (int j = 0; j < V; ++j) {
-                    const int4 q = d4[j];
-                    if constexpr (sizeof(MemT) == 4) s += q.x + q.y + q.z + q.w;
-                    else {
-                        const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
-                        s += (MemT)(l.x + l.y);
-                    }
-                }
-                MemT run = warp_inclusive_sum(s, lane) - s;
                 MemT peak = 0;
-                for (int j = 0; j < V; ++j) {
-                    const int4 q = d4[j];
-                    if constexpr (sizeof(MemT) == 4) {
-                        run += q.x; peak = max(peak, run);
-                        run += q.y; peak = max(peak, run);
-                        run += q.z; peak = max(peak, run);
-                        run += q.w; peak = max(peak, run);
-                    } else {
-                        const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
-                        run += (MemT)l.x; peak = run > peak ? run : peak;
-                        run += (MemT)l.y; peak = run > peak ? run : peak;
+                if (kRegVecs > 0 && V <= kRegVecs) {
+                    int4 q[kRegVecs > 0 ? kRegVecs : 1];
+                    int32_t s = 0;
+#pragma unroll
+                    for (int j = 0; j < kRegVecs; ++j) {
+                        q[j] = make_int4(0, 0, 0, 0);
+                        if (j < V) q[j] = d4[j];
+                        s += q[j].x + q[j].y + q[j].z + q[j].w;
+                    }
+                    int32_t run = warp_inclusive_sum(s, lane) - s;
+                    int32_t pk = 0;
+#pragma unroll
+                    for (int j = 0; j < kRegVecs; ++j) {
+                        run += q[j].x; pk = max(pk, run);
+                        run += q[j].y; pk = max(pk, run);
+                        run += q[j].z; pk = max(pk, run);
+                        run += q[j].w; pk = max(pk, run);
+                    }
+                    peak = (MemT)pk;
+                } else {
+                    MemT s = 0;
+                    for (int j = 0; j < V; ++j) {
+                        const int4 q = d4[j];
+                        if constexpr (sizeof(MemT) == 4) s += q.x + q.y + q.z + q.w;
+                        else {
+                            const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
+                            s += (MemT)(l.x + l.y);
+                        }
+                    }
+                    MemT run = warp_inclusive_sum(s, lane) - s;
+                    for (int j = 0; j < V; ++j) {
+                        const int4 q = d4[j];
+                        if constexpr (sizeof(MemT) == 4) {
+                            run += q.x; peak = max(peak, run);
+                            run += q.y; peak = max(peak, run);
+                            run += q.z; peak = max(peak, run);
+                            run += q.w; peak = max(peak, run);
+                        } else {
+                            const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
+                            run += (MemT)l.x; peak = run > peak ? run : peak;
+                            run += (MemT)l.y; peak = run > peak ? run : peak;
+                        }
                     }
                 }
                 out_pk = (int64_t)warp_max_t(peak);
