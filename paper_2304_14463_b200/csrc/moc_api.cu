@@ -45,7 +45,7 @@ struct Plan {
     // fast path for C <= 2: a warp per sequence, graph staged in shared memory
     bool pair = false;
     PairFn pair_fn = nullptr;
-    uint32_t rec_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
+    uint32_t rec_bytes = 0, w_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
 };
 
 }  // namespace
@@ -65,10 +65,11 @@ struct moc_graph {
     int32_t* d_m32 = nullptr;
     int32_t want_G = 0, want_gpc = 0;
     // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
-    int32_t sell_len = 0, n_slices = 0;
+    int32_t sell_len = 0, n_tiles = 0;
     void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
     void* d_rec64 = nullptr;
-    uint16_t* d_sell = nullptr;
+    int64_t* d_wslot = nullptr;
+    uint32_t* d_sell = nullptr;
     uint32_t* d_tile = nullptr;
     // grow-only scratch; mutable because evaluation takes a const handle
     mutable Plan plan_eval, plan_profile;
@@ -141,10 +142,11 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         const size_t msz = pl.wide ? 8 : 4, per_vec = 16 / msz;
         const size_t nvec_d = (t_max + 1 + per_vec - 1) / per_vec;
         const size_t v_max = ((nvec_d + 31) / 32) | 1;
-        const size_t rec_b = align16((pl.wide ? sizeof(moc::NodeRec<int64_t>) : sizeof(moc::NodeRec<int32_t>)) * n),
-                     col_b = align16(4 * (size_t)g->n_slices), jds_b = align16(2 * (size_t)g->sell_len),
+        const size_t rec_b = (pl.wide ? sizeof(moc::NodeRec<int64_t>) : sizeof(moc::NodeRec<int32_t>)) * 64 * (size_t)g->n_tiles,
+                     col_b = align16(4 * (size_t)g->n_tiles), jds_b = align16(4 * (size_t)g->sell_len),
                      word_b = align16(4 * (n + 1)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
-        const size_t graph_b = rec_b + col_b + jds_b, warp_b = word_b + delta_b;
+        const size_t w_b = 8 * 64 * (size_t)g->n_tiles;
+        const size_t graph_b = rec_b + w_b + col_b + jds_b, warp_b = word_b + moc::kPairWordTail + delta_b;
         PairFn fn = pl.wide ? (PairFn)moc::eval_pair_kernel<int64_t> : (PairFn)moc::eval_pair_kernel<int32_t>;
         int best_wpb = 0, best_warps = 0, best_nb = 0;
         const int cand[4] = {16, 12, 8, 4};
@@ -166,7 +168,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             pl.block = 32 * best_wpb;
             pl.smem = graph_b + best_wpb * warp_b;
             pl.grid = g->sm_count * best_nb;
-            pl.rec_bytes = (uint32_t)rec_b; pl.tile_bytes = (uint32_t)col_b;
+            pl.rec_bytes = (uint32_t)rec_b; pl.w_bytes = (uint32_t)w_b; pl.tile_bytes = (uint32_t)col_b;
             pl.sell_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
             cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
             if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
@@ -278,28 +280,22 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
     const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
     moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
     ++g_launches;
-    // the evaluation kernel may begin (stage the graph, set up shared memory) while the offsets
-    // kernel still runs; it waits for the offsets inside
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)pl.block);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     if (pl.pair) {
         moc::PairParams q{};
         q.n = g->n;
         q.sell_len = g->sell_len;
-        q.n_slices = g->n_slices;
+        q.n_tiles = g->n_tiles;
+        q.sum_bias = (uint32_t)(64 * g->n_tiles - g->n);
         q.max_T = g->C * g->n;
         q.rec = pl.wide ? g->d_rec64 : g->d_rec32;
+        q.wslot = g->d_wslot;
         q.sell = g->d_sell;
         q.tile = g->d_tile;
-        q.w = g->d_w;
         q.base_dur = g->sum_w;
         q.seqs = seqs;
         q.lens = lens;
@@ -309,7 +305,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
         q.out_peak = out_peak;
         q.out_dur = out_dur;
         q.out_status = out_feasible;
-        q.rec_bytes = pl.rec_bytes; q.tile_bytes = pl.tile_bytes; q.sell_bytes = pl.sell_bytes;
+        q.rec_bytes = pl.rec_bytes; q.w_bytes = pl.w_bytes; q.tile_bytes = pl.tile_bytes; q.sell_bytes = pl.sell_bytes;
         q.word_bytes = pl.word_bytes; q.delta_bytes = pl.delta_bytes;
         MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.pair_fn, q));
     } else {
@@ -436,49 +432,93 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     up((void**)&g->d_w, w, (size_t)n * 8);
     up((void**)&g->d_m64, m, (size_t)n * 8);
     up((void**)&g->d_m32, m32.data(), (size_t)n * 4);
-    if (n <= 16383) {
-        // successor lists as a sliced ELL matrix: nodes sorted by out-degree (descending, ties by
-        // id) in slices of 32; slice s is a [degree of its first node][32] tile of byte offsets
-        // 4*successor, padded with 4*n (a dummy word).  Skipped when padding would more than
-        // double the storage (a few very high degrees): such graphs use the general kernel.
+    if (n <= 16000) {
+        // Layout for the warp-per-sequence kernel.  Lane l serves the nodes with id = l (mod 32);
+        // each residue class is sorted by out-degree (descending, ties by id); half j holds the
+        // j-th node of every class, a tile is two halves.  A tile stores, row by row, the word
+        // offsets (4 * id) of its nodes' successors, two halves packed per 32-bit entry, padded with
+        // the offset of a dummy word (4 * n).  Within a half the order of each node's successors
+        // is chosen greedily so that the 32 words a row touches fall in different banks where
+        // possible.  Skipped when padding would more than double the storage (a few very high
+        // degrees): such graphs use the general kernel.
         try {
-            std::vector<int32_t> order((size_t)n);
-            for (int32_t v = 0; v < n; ++v) order[v] = v;
             auto deg = [&](int32_t v) { return succ_start[v + 1] - succ_start[v]; };
-            std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
-            const int32_t n_slices = (n + 31) / 32;
+            const int32_t n_halves = 2 * ((n + 63) / 64), n_tiles = n_halves / 2;
+            std::vector<int32_t> slot((size_t)n_halves * 32, -1);  // node at (half, lane) or -1
+            for (int32_t l = 0; l < 32; ++l) {
+                std::vector<int32_t> cls;
+                for (int32_t v = l; v < n; v += 32) cls.push_back(v);
+                std::stable_sort(cls.begin(), cls.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
+                for (size_t j = 0; j < cls.size(); ++j) slot[j * 32 + l] = cls[j];
+            }
+            std::vector<int32_t> rows((size_t)n_tiles, 0);
             int64_t sell_len = 0;
-            for (int32_t s = 0; s < n_slices; ++s) sell_len += 32 * (int64_t)deg(order[32 * s]);
-            if (sell_len <= 2 * ne + 32 * 64 && sell_len < (1 << 18)) {
-                std::vector<uint32_t> tile((size_t)n_slices);
-                std::vector<moc::NodeRec<int32_t>> rec32((size_t)n);
-                std::vector<moc::NodeRec<int64_t>> rec64((size_t)n);
-                std::vector<uint16_t> sell((size_t)std::max<int64_t>(sell_len, 1), (uint16_t)(4 * n));
-                for (int32_t i = 0; i < n; ++i) {
-                    const uint32_t nd = 4u * (uint32_t)order[i] | ((uint32_t)deg(order[i]) << 16);
-                    rec32[i].nd = nd;
-                    rec32[i].m = m32[order[i]];
-                    rec64[i].nd = nd;
-                    rec64[i].pad = 0;
-                    rec64[i].m = m[order[i]];
+            for (int32_t d = 0; d < n_tiles; ++d) {
+                for (int32_t s = 0; s < 64; ++s)
+                    if (slot[(size_t)d * 64 + s] >= 0) rows[d] = std::max(rows[d], deg(slot[(size_t)d * 64 + s]));
+                sell_len += 32 * (int64_t)rows[d];
+            }
+            int32_t max_rows = 0;
+            for (int32_t d = 0; d < n_tiles; ++d) max_rows = std::max(max_rows, rows[d]);
+            if (sell_len <= 2 * ne + 4096 && sell_len < (1 << 20) && max_rows < (1 << 12)) {
+                const uint32_t word_b = (uint32_t)align16(4 * ((size_t)n + 1));
+                const uint32_t dummy = 4u * (uint32_t)n;
+                std::vector<uint32_t> tile((size_t)n_tiles);
+                std::vector<moc::NodeRec<int32_t>> rec32((size_t)n_halves * 32);
+                std::vector<moc::NodeRec<int64_t>> rec64((size_t)n_halves * 32);
+                std::vector<int64_t> wslot((size_t)n_halves * 32);
+                std::vector<uint32_t> sell((size_t)std::max<int64_t>(sell_len, 1), dummy | (dummy << 16));
+                for (size_t r = 0; r < slot.size(); ++r) {
+                    const int32_t v = slot[r];
+                    const uint32_t nd = v >= 0 ? (4u * (uint32_t)v | ((uint32_t)deg(v) << 16)) : word_b;
+                    rec32[r].nd = nd;
+                    rec32[r].m = v >= 0 ? m32[v] : 0;
+                    wslot[r] = v >= 0 ? w[v] : 0;
+                    rec64[r].nd = nd;
+                    rec64[r].pad = 0;
+                    rec64[r].m = v >= 0 ? m[v] : 0;
                 }
                 uint32_t pos = 0;
-                for (int32_t s = 0; s < n_slices; ++s) {
-                    const int32_t rows = deg(order[32 * s]);
-                    tile[s] = pos | ((uint32_t)rows << 18);
-                    for (int32_t l = 0; l < 32 && 32 * s + l < n; ++l) {
-                        const int32_t u = order[32 * s + l];
-                        for (int32_t k = 0; k < deg(u); ++k)
-                            sell[pos + 32 * k + l] = (uint16_t)(4 * succ[succ_start[u] + k]);
+                std::vector<std::vector<int32_t>> rem(32);
+                for (int32_t d = 0; d < n_tiles; ++d) {
+                    tile[d] = pos | ((uint32_t)rows[d] << 20);
+                    for (int32_t h = 0; h < 2; ++h) {
+                        std::vector<int32_t> lanes;
+                        for (int32_t l = 0; l < 32; ++l) {
+                            const int32_t v = slot[((size_t)2 * d + h) * 32 + l];
+                            rem[l].clear();
+                            if (v >= 0) rem[l].assign(succ.begin() + succ_start[v], succ.begin() + succ_start[v + 1]);
+                            lanes.push_back(l);
+                        }
+                        for (int32_t k = 0; k < rows[d]; ++k) {
+                            int used[32] = {0};
+                            std::stable_sort(lanes.begin(), lanes.end(),
+                                             [&](int32_t x, int32_t y) { return rem[x].size() > rem[y].size(); });
+                            for (int32_t l : lanes) {
+                                if (rem[l].empty()) continue;  // stays the dummy
+                                const bool forced = (int32_t)rem[l].size() >= rows[d] - k;
+                                int pick = -1;
+                                for (size_t c = 0; c < rem[l].size(); ++c)
+                                    if (!used[rem[l][c] & 31]) { pick = (int)c; break; }
+                                if (pick < 0 && !forced) continue;  // wait for a row where its bank is free
+                                if (pick < 0) pick = 0;
+                                const uint32_t off = 4u * (uint32_t)rem[l][pick];
+                                used[rem[l][pick] & 31]++;
+                                rem[l].erase(rem[l].begin() + pick);
+                                uint32_t& e = sell[pos + 32 * (uint32_t)k + l];
+                                e = h == 0 ? ((e & 0xFFFF0000u) | off) : ((e & 0x0000FFFFu) | (off << 16));
+                            }
+                        }
                     }
-                    pos += 32 * (uint32_t)rows;
+                    pos += 32 * (uint32_t)rows[d];
                 }
                 g->sell_len = (int32_t)sell_len;
-                g->n_slices = n_slices;
-                up(&g->d_rec32, rec32.data(), (size_t)n * sizeof(rec32[0]));
-                up(&g->d_rec64, rec64.data(), (size_t)n * sizeof(rec64[0]));
-                up((void**)&g->d_sell, sell.data(), (size_t)sell_len * 2);
-                up((void**)&g->d_tile, tile.data(), (size_t)n_slices * 4);
+                g->n_tiles = n_tiles;
+                up(&g->d_rec32, rec32.data(), rec32.size() * sizeof(rec32[0]));
+                up(&g->d_rec64, rec64.data(), rec64.size() * sizeof(rec64[0]));
+                up((void**)&g->d_wslot, wslot.data(), wslot.size() * 8);
+                up((void**)&g->d_sell, sell.data(), (size_t)sell_len * 4);
+                up((void**)&g->d_tile, tile.data(), (size_t)n_tiles * 4);
             }
         } catch (const std::bad_alloc&) {
             moc_graph_destroy(g);
@@ -526,6 +566,7 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_m32);
     cudaFree(g->d_rec32);
     cudaFree(g->d_rec64);
+    cudaFree(g->d_wslot);
     cudaFree(g->d_sell);
     cudaFree(g->d_tile);
     cudaFree(g->d_offs);

@@ -54,14 +54,6 @@ template <typename PosT> struct PosNone;
 template <> struct PosNone<uint16_t> { static constexpr uint32_t value = 0xFFFFu; };
 template <> struct PosNone<int32_t> { static constexpr uint32_t value = 0x7FFFFFFFu; };
 
-// Waits until the kernel launched before this one in the stream has finished and its writes are
-// visible (no-op unless this kernel was launched with programmatic stream serialization).
-__device__ __forceinline__ void wait_for_previous_kernel() {
-#if __CUDA_ARCH__ >= 900
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
-}
-
 template <int G>
 __device__ __forceinline__ void group_sync(int bar_id) {
     if constexpr (G == 32) {
@@ -330,7 +322,6 @@ __device__ __forceinline__ void eval_one(const EvalParams& p, const int b, const
 template <int G, typename MemT, int CP, bool kProfile>
 __global__ void __launch_bounds__(1024) eval_shared_kernel(const EvalParams p) {
     extern __shared__ __align__(16) char smem[];
-    wait_for_previous_kernel();
     const int gpc = blockDim.x / G;
     const int gi = threadIdx.x / G, tid = threadIdx.x % G;
     char* state = smem + (size_t)gi * p.group_bytes;
@@ -344,7 +335,6 @@ __global__ void __launch_bounds__(1024) eval_shared_kernel(const EvalParams p) {
 template <int CP, bool kProfile>
 __global__ void __launch_bounds__(1024) eval_global_kernel(const EvalParams p) {
     char* state = p.gstate + (size_t)blockIdx.x * p.group_bytes;
-    wait_for_previous_kernel();
     for (int b = blockIdx.x; b < p.B; b += gridDim.x)
         eval_one<1024, int64_t, int32_t, CP, kProfile>(p, b, threadIdx.x, 0, state);
 }
@@ -352,25 +342,42 @@ __global__ void __launch_bounds__(1024) eval_global_kernel(const EvalParams p) {
 // offs = exclusive prefix sum of max(lens, 0); offs[B] = total.
 // Block j owns elements [j*kOffsTile, (j+1)*kOffsTile): it first adds up everything in front of its
 // tile (redundantly with the other blocks -- B is small, and this needs no cross-block handshake),
-// then scans its own tile.  The dependent evaluation kernel may start its prologue at once.
-constexpr int kOffsThreads = 512;
+// then scans its own tile.
+constexpr int kOffsThreads = 256;
 constexpr int kOffsPer = 4;
 constexpr int kOffsTile = kOffsThreads * kOffsPer;
 
 __global__ void __launch_bounds__(kOffsThreads) offsets_kernel(const int32_t* __restrict__ lens, int32_t B,
                                                                 int64_t* __restrict__ offs) {
-#if __CUDA_ARCH__ >= 900
-    asm volatile("griddepcontrol.launch_dependents;");
-#endif
     __shared__ int64_t wsum[kOffsThreads / 32];
     __shared__ int64_t wtot[kOffsThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t tile0 = (int64_t)blockIdx.x * kOffsTile;
-    // ---- sum of everything before the tile
+    // ---- sum of everything before the tile (16-byte loads, several in flight per thread)
     int64_t s = 0;
-    for (int64_t i = tid; i < tile0; i += kOffsThreads) {
-        const int32_t v = __ldg(lens + i);
-        s += v > 0 ? v : 0;
+    if ((reinterpret_cast<uintptr_t>(lens) & 15) == 0) {
+        const int4* l4 = reinterpret_cast<const int4*>(lens);
+        const int64_t n4 = tile0 >> 2;  // the tile size is a multiple of 4
+        int64_t s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+        int64_t i = tid;
+        for (; i + 3 * kOffsThreads < n4; i += 4 * kOffsThreads) {
+            const int4 a = __ldg(l4 + i), b = __ldg(l4 + i + kOffsThreads), c = __ldg(l4 + i + 2 * kOffsThreads),
+                       d = __ldg(l4 + i + 3 * kOffsThreads);
+            s0 += (int64_t)max(a.x, 0) + max(a.y, 0) + max(a.z, 0) + max(a.w, 0);
+            s1 += (int64_t)max(b.x, 0) + max(b.y, 0) + max(b.z, 0) + max(b.w, 0);
+            s2 += (int64_t)max(c.x, 0) + max(c.y, 0) + max(c.z, 0) + max(c.w, 0);
+            s3 += (int64_t)max(d.x, 0) + max(d.y, 0) + max(d.z, 0) + max(d.w, 0);
+        }
+        for (; i < n4; i += kOffsThreads) {
+            const int4 a = __ldg(l4 + i);
+            s0 += (int64_t)max(a.x, 0) + max(a.y, 0) + max(a.z, 0) + max(a.w, 0);
+        }
+        s = s0 + s1 + s2 + s3;
+    } else {
+        for (int64_t i = tid; i < tile0; i += kOffsThreads) {
+            const int32_t v = __ldg(lens + i);
+            s += v > 0 ? v : 0;
+        }
     }
     s = warp_sum(s);
     if (lane == 0) wtot[warp] = s;

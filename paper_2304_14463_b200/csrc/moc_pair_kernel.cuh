@@ -4,12 +4,16 @@
 //
 // Representation.  Positions are 1-based and 16 bits wide; 0 means "no copy".  Each node owns one
 // 32-bit word holding its (at most two) positions, so a consumer reads both copies of a
-// predecessor/successor with one load.  The successor lists are stored as a sliced ELL matrix:
-// nodes are sorted by out-degree (descending) and cut into slices of 32; slice s is a dense
-// [degree of its first node][32] tile whose row k holds the k-th successor of each of its nodes, as
-// the byte offset of that successor's word, padded with the offset of a dummy word that stays zero.
-// Lanes read consecutive entries, every lane of a warp runs the same trip count, and the padding
-// is neutral for the maxima and minima taken over the successors.
+// predecessor/successor with one load.  Lane l of a warp works on the nodes with id = l (mod 32):
+// a node's word then sits in bank l, so the lanes' reads of their own words never collide.  The
+// nodes of each residue class are sorted by out-degree (descending); "half" j holds the j-th node
+// of every class and a tile is two consecutive halves, so a lane treats two nodes per tile.  The
+// successor lists are stored per tile as a dense [rows][32] matrix of 32-bit entries: entry
+// (k, l) packs the word offsets of the k-th successor of lane l's two nodes, 16 bits each; rows =
+// largest out-degree in the tile; missing successors point at a dummy word that stays zero, which
+// is neutral for the maxima and minima taken over the successors.  Every lane of a warp runs the
+// same trip count.  Node slots beyond the last node of a class read a word that holds the
+// constant 1 and carry m = w = 0, so they need no special case.
 //
 // Stages for one sequence seq[0..T) (paper: Section 2, Eqs. 1-8):
 //   1. occurrence words   step t exchanges t+1 into the low half of its node's word and moves the
@@ -37,13 +41,14 @@ namespace moc {
 
 struct PairParams {
     int32_t n;
-    int32_t sell_len;          // entries of the sliced ELL matrix
-    int32_t n_slices;          // ceil(n / 32)
+    int32_t n_tiles;           // tiles of 64 node slots (two halves of 32)
+    int32_t sell_len;          // 32-bit entries of the successor tiles
     int32_t max_T;             // C * n
-    const void* rec;           // n node records (NodeRec<MemT>) in out-degree order
-    const uint16_t* sell;      // sell_len byte offsets (4 * successor id, 4 * n = dummy)
-    const uint32_t* tile;      // n_slices: first entry of the slice | rows of the slice << 18
-    const int64_t* w;          // n durations by node id
+    uint32_t sum_bias;         // number of empty node slots (each reads a word holding 1)
+    const void* rec;           // 64 * n_tiles node records (NodeRec<MemT>), slot = half * 32 + lane
+    const int64_t* wslot;      // 64 * n_tiles durations, same slots
+    const uint32_t* sell;      // sell_len entries: successor word offsets of the two halves, 16 bits each
+    const uint32_t* tile;      // n_tiles: first entry of the tile | rows of the tile << 20
     int64_t base_dur;          // sum of all w
     const int32_t* seqs;
     const int32_t* lens;
@@ -54,41 +59,53 @@ struct PairParams {
     int64_t* out_dur;
     int32_t* out_status;
     // shared-memory layout, bytes (multiples of 16)
-    uint32_t rec_bytes, tile_bytes, sell_bytes;  // graph, once per block
-    uint32_t word_bytes, delta_bytes;                  // per warp
+    uint32_t rec_bytes, w_bytes, tile_bytes, sell_bytes;  // graph, once per block
+    uint32_t word_bytes, delta_bytes;            // per warp; 16 bytes after the words hold the constant 1
 };
 
 constexpr int kPairDeltaFront = 16;  // bytes in front of delta[0]: lands writes of absent nodes
+constexpr int kPairWordTail = 16;    // bytes after the words: the word read by empty node slots
 
 __device__ __forceinline__ int64_t warp_sum64(int64_t v) {
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
     return v;
 }
-// per-halfword unsigned max / min of two packed 16-bit pairs (one instruction on sm_90 and later)
+__device__ __forceinline__ int32_t warp_max_t(int32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
+__device__ __forceinline__ int64_t warp_max_t(int64_t v) { return warp_max(v); }
+
+// per-halfword unsigned max of two packed 16-bit pairs (one instruction on sm_90 and later)
 __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
-__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
+
+// ---- shared-memory accesses by 32-bit shared address
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
 }
-__device__ __forceinline__ uint32_t add_u16x2(uint32_t a, uint32_t b) {  // per halfword, wraps
-    uint32_t d;
-    asm("add.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ uint32_t exch_shared(uint32_t addr, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void red_add_shared(uint32_t addr, int32_t v) {
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_add_shared(uint32_t addr, int64_t v) {
+    asm volatile("red.shared.add.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 
-// Node record: byte offset of the node's word (4 * id) | out-degree << 16, and its output size.
+// Node record: byte offset of the node's word | out-degree << 16, and the output size.
 template <typename MemT> struct NodeRec;
 template <> struct __align__(8) NodeRec<int32_t> { uint32_t nd; int32_t m; };
 template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; int64_t m; };
-
-__device__ __forceinline__ int32_t warp_max_t(int32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
-__device__ __forceinline__ int64_t warp_max_t(int64_t v) { return warp_max(v); }
 
 template <typename MemT>
 __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
@@ -96,34 +113,47 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     using Rec = NodeRec<MemT>;
     // ---- graph -> shared memory, once per block
     Rec* s_rec = reinterpret_cast<Rec*>(smem);
-    uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem + p.rec_bytes);
-    uint16_t* s_sell = reinterpret_cast<uint16_t*>(smem + p.rec_bytes + p.tile_bytes);
-    const uint32_t graph_bytes = p.rec_bytes + p.tile_bytes + p.sell_bytes;
+    int64_t* s_w = reinterpret_cast<int64_t*>(smem + p.rec_bytes);
+    uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem + p.rec_bytes + p.w_bytes);
+    uint32_t* s_sell = reinterpret_cast<uint32_t*>(smem + p.rec_bytes + p.w_bytes + p.tile_bytes);
+    const uint32_t graph_bytes = p.rec_bytes + p.w_bytes + p.tile_bytes + p.sell_bytes;
     {
-        const Rec* grec = reinterpret_cast<const Rec*>(p.rec);
-        for (int i = threadIdx.x; i < p.n; i += blockDim.x) s_rec[i] = grec[i];
-        for (int i = threadIdx.x; i < p.n_slices; i += blockDim.x) s_tile[i] = __ldg(&p.tile[i]);
+        const int4* g4 = reinterpret_cast<const int4*>(p.rec);
+        int4* s4 = reinterpret_cast<int4*>(s_rec);
+        const int n4 = (int)sizeof(Rec) * 64 * p.n_tiles / 16;
+        for (int i = threadIdx.x; i < n4; i += blockDim.x) s4[i] = __ldg(&g4[i]);
+        for (int i = threadIdx.x; i < 64 * p.n_tiles; i += blockDim.x) s_w[i] = __ldg(&p.wslot[i]);
+        for (int i = threadIdx.x; i < p.n_tiles; i += blockDim.x) s_tile[i] = __ldg(&p.tile[i]);
         for (int i = threadIdx.x; i < p.sell_len; i += blockDim.x) s_sell[i] = __ldg(&p.sell[i]);
     }
-    __syncthreads();
-    wait_for_previous_kernel();  // the packing offsets come from the kernel launched just before
-
     const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     // broadcast from lane 0 so that the compiler knows the warp index is uniform across the warp
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
-    char* ws = smem + graph_bytes + (size_t)warp * (p.word_bytes + p.delta_bytes);
+    char* ws = smem + graph_bytes + (size_t)warp * (p.word_bytes + kPairWordTail + p.delta_bytes);
     uint32_t* word = reinterpret_cast<uint32_t*>(ws);
-    uint16_t* word16 = reinterpret_cast<uint16_t*>(ws);
-    char* delta_base = ws + p.word_bytes;                          // includes the front pad
-    MemT* delta = reinterpret_cast<MemT*>(delta_base + kPairDeltaFront);
+    char* delta_base = ws + p.word_bytes + kPairWordTail;          // includes the front pad
+    const uint32_t wa = (uint32_t)__cvta_generic_to_shared(word);
+    const uint32_t da = (uint32_t)__cvta_generic_to_shared(delta_base) + kPairDeltaFront;  // &delta[0]
+    if (lane == 0) *reinterpret_cast<uint32_t*>(ws + p.word_bytes) = 1u;   // read by empty node slots
+    __syncthreads();
+
     const int n = p.n;
     const int n_warps = gridDim.x * wpb;
     constexpr int kPerVec = 16 / (int)sizeof(MemT);  // delta entries per 16-byte vector
+    constexpr int kShift = sizeof(MemT) == 4 ? 2 : 3;
     constexpr int kRegVecs = sizeof(MemT) == 4 ? 7 : 0;  // scan keeps up to this many vectors per lane in registers
 
-    for (int b = blockIdx.x * wpb + warp; b < p.B; b += n_warps) {
-        const int64_t off = p.offs[b];
-        const int32_t T = p.lens[b];
+    int b = blockIdx.x * wpb + warp;
+    int64_t off = 0;
+    int32_t T = 0;
+    if (b < p.B) { off = __ldg(&p.offs[b]); T = __ldg(&p.lens[b]); }
+    while (b < p.B) {
+        // fetch the next sequence's place early: its latency hides behind this sequence's work
+        const int b_next = b + n_warps;
+        int64_t off_next = 0;
+        int32_t T_next = 0;
+        if (b_next < p.B) { off_next = __ldg(&p.offs[b_next]); T_next = __ldg(&p.lens[b_next]); }
+
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;
         if (T >= n && T <= p.max_T) {
@@ -147,8 +177,9 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 const int nvec = (T + a + 3) >> 2;
                 auto put = [&](int node, uint32_t t1) {
                     if ((unsigned)node < (unsigned)n) {
-                        const uint32_t old = atomicExch(&word[node], t1);
-                        if (old) word16[2 * node + 1] = (uint16_t)old;
+                        const uint32_t addr = wa + 4u * (uint32_t)node;
+                        const uint32_t old = exch_shared(addr, t1);
+                        if (old) sts_u16(addr + 2, old);
                     }
                 };
                 // vectors that lie completely inside the row
@@ -177,60 +208,67 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             }
             __syncwarp();
 
-            // ---- stage 2 and the scatter of stage 3: one lane per node, slices in out-degree order
+            // ---- stage 2 and the scatter of stage 3: two node slots per lane and tile
             uint32_t vmin = 0xFFFFFFFFu, vsum = 0;
-            bool dep = false;
+            uint32_t depw = 0;
             int64_t dur_extra = 0;
-            for (int i0 = 0, sl = 0; i0 < n; i0 += 32, ++sl) {
-                const int i = i0 + lane;
-                const bool live = i < n;
-                Rec rec;
-                rec.nd = 4u * (uint32_t)n;  // lanes past the last node look at the dummy word
-                rec.m = 0;
-                if (live) rec = s_rec[i];
-                const uint32_t own = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(word) + (rec.nd & 0xFFFFu));
-                const uint32_t lo = own & 0xFFFFu, hi = own >> 16;
-                const bool dbl = hi != 0;
-                const uint32_t hh = dbl ? hi : lo;
-                const uint32_t a = min(lo, hh), bpos = max(lo, hh);
-                const uint32_t nbb = ((0x10000u - bpos) & 0xFFFFu) * 0x10001u;   // -b in both halves
-                // successors of the slice: uniform trip count, padded entries read the dummy word
-                const uint32_t tl = __shfl_sync(0xFFFFFFFFu, s_tile[sl], 0);
-                const uint16_t* pj = s_sell + (tl & 0x3FFFFu) + lane;
-                const int rows = (int)(tl >> 18);
-                uint32_t F = 0, D = 0xFFFFFFFFu, G = 0;
-#pragma unroll 4
-                for (int k = 0; k < rows; ++k) {
-                    const uint32_t v4 = pj[k * 32];
-                    const uint32_t r = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(word) + v4);
-                    F = max_u16x2(F, r);
-                    D = min_u16x2(D, r - 0x00010001u);   // empty half -> 0xFFFF
-                    G = max_u16x2(G, add_u16x2(r, nbb));
+            for (int d = 0; d < p.n_tiles; ++d) {
+                Rec rec[2];
+                uint32_t lo[2], hi[2], a[2], bpos[2], nbb[2], F[2], D[2], G[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    rec[h] = s_rec[(2 * d + h) * 32 + lane];
+                    const uint32_t own = lds_u32(wa + (rec[h].nd & 0xFFFFu));
+                    lo[h] = own & 0xFFFFu;
+                    hi[h] = own >> 16;
+                    const uint32_t hh = hi[h] ? hi[h] : lo[h];
+                    a[h] = min(lo[h], hh);
+                    bpos[h] = max(lo[h], hh);
+                    nbb[h] = ((0u - bpos[h]) & 0xFFFFu) * 0x10001u;   // -b mod 2^16 in both halves
+                    F[h] = 0; D[h] = 0xFFFFFFFFu; G[h] = 0;
                 }
-                if (live) {
-                    const uint32_t deg = rec.nd >> 16;
-                    vmin = min(vmin, lo);
-                    vsum += lo + hi;
-                    const uint32_t Fm = max(F & 0xFFFFu, F >> 16);
-                    const uint32_t Dm = min(D & 0xFFFFu, D >> 16);
-                    if (deg != 0 && Dm + 1 < a) dep = true;   // a successor copy before the first copy of u
-                    const uint32_t fb = deg != 0 ? max(Fm, bpos) : (uint32_t)T;
-                    atomic_add_mem(&delta[(int)bpos - 1], rec.m);
-                    atomic_add_mem(&delta[fb], (MemT)(-rec.m));
-                    if (dbl) {
-                        // latest successor copy h with a < h < b, if any: (h - b) mod 2^16 is the largest
-                        const uint32_t h = (max(G & 0xFFFFu, G >> 16) + bpos) & 0xFFFFu;
-                        const uint32_t fa = (h - 1u < bpos - 1u) ? h : a;
-                        atomic_add_mem(&delta[(int)a - 1], rec.m);
-                        atomic_add_mem(&delta[fa], (MemT)(-rec.m));
-                        dur_extra += __ldg(&p.w[(rec.nd & 0xFFFFu) >> 2]);
+                // successors of the tile: uniform trip count, padded entries read the dummy word
+                const uint32_t tl = __shfl_sync(0xFFFFFFFFu, s_tile[d], 0);
+                const uint32_t* pj = s_sell + (tl & 0xFFFFFu) + lane;
+                const int rows = (int)(tl >> 20);
+#pragma unroll 2
+                for (int k = 0; k < rows; ++k) {
+                    const uint32_t e = pj[k * 32];
+                    const uint32_t r0 = lds_u32(wa + (e & 0xFFFFu));
+                    const uint32_t r1 = lds_u32(wa + (e >> 16));
+                    F[0] = max_u16x2(F[0], r0);
+                    F[1] = max_u16x2(F[1], r1);
+                    D[0] = __viaddmin_u16x2(r0, 0xFFFFFFFFu, D[0]);   // min(r - 1): empty half -> 0xFFFF
+                    D[1] = __viaddmin_u16x2(r1, 0xFFFFFFFFu, D[1]);
+                    G[0] = __viaddmax_u16x2(r0, nbb[0], G[0]);        // max(r - b)
+                    G[1] = __viaddmax_u16x2(r1, nbb[1], G[1]);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t deg = rec[h].nd >> 16;
+                    vmin = min(vmin, lo[h]);
+                    vsum += lo[h] + hi[h];
+                    const uint32_t Fm = max(F[h] & 0xFFFFu, F[h] >> 16);
+                    const uint32_t Dm = min(D[h] & 0xFFFFu, D[h] >> 16);
+                    // a successor copy before the first copy of u (deg = 0: D stays 0xFFFF)
+                    depw |= (Dm + 1 < a[h]) ? 1u : 0u;
+                    const uint32_t fb = deg != 0 ? max(Fm, bpos[h]) : (uint32_t)T;
+                    red_add_shared(da + ((bpos[h] - 1u) << kShift), rec[h].m);
+                    red_add_shared(da + (fb << kShift), (MemT)(-rec[h].m));
+                    if (hi[h] != 0) {
+                        dur_extra += s_w[(2 * d + h) * 32 + lane];
+                        // latest successor copy x with a < x < b, if any: (x - b) mod 2^16 is the largest
+                        const uint32_t x = (max(G[h] & 0xFFFFu, G[h] >> 16) + bpos[h]) & 0xFFFFu;
+                        const uint32_t fa = (x - 1u < bpos[h] - 1u) ? x : a[h];
+                        red_add_shared(da + ((a[h] - 1u) << kShift), rec[h].m);
+                        red_add_shared(da + (fa << kShift), (MemT)(-rec[h].m));
                     }
                 }
             }
             vmin = __reduce_min_sync(0xFFFFFFFFu, vmin);
             vsum = __reduce_add_sync(0xFFFFFFFFu, vsum);
-            const bool well_formed = vmin != 0 && vsum == (uint32_t)T * ((uint32_t)T + 1u) / 2u;
-            dep = __any_sync(0xFFFFFFFFu, dep);
+            const bool well_formed = vmin != 0 && vsum == (uint32_t)T * ((uint32_t)T + 1u) / 2u + p.sum_bias;
+            const bool dep = __any_sync(0xFFFFFFFFu, depw != 0);
             __syncwarp();
 
             if (!well_formed) {
@@ -240,7 +278,7 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 out_du = p.base_dur + warp_sum64(dur_extra);
             } else {
                 // ---- stage 3 + 4: prefix sum and running maximum; lane owns V consecutive vectors
-                const int4* d4 = reinterpret_cast<const int4*>(delta) + lane * V;
+                const int4* d4 = reinterpret_cast<const int4*>(delta_base + kPairDeltaFront) + lane * V;
                 MemT peak = 0;
                 if (kRegVecs > 0 && V <= kRegVecs) {
                     int4 q[kRegVecs > 0 ? kRegVecs : 1];
@@ -297,6 +335,9 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             p.out_dur[b] = out_du;
             p.out_status[b] = out_st;
         }
+        b = b_next;
+        off = off_next;
+        T = T_next;
     }
 }
 
