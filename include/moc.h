@@ -167,6 +167,15 @@ int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t
  */
 int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t sequences_per_block);
 
+/*
+ * Measurement hook: while set, every moc_eval_batch on this handle records `before` right before
+ * and `after` right after its evaluation kernel (the dominant kernel; the offsets kernel lies
+ * outside the pair), on the stream of the call.  Both are cudaEvent_t created by the caller with
+ * timing enabled; pass NULL, NULL to switch the hook off.  The caller reads the elapsed time after
+ * synchronising.  Costs two event records per call, so leave it off outside of measurements.
+ */
+int moc_graph_set_timing_events(moc_graph* g, void* before, void* after);
+
 /* Number of kernels the most recent moc_eval_batch / moc_mem_profile on this thread launched. */
 int moc_last_launch_count(void);
 

@@ -18,7 +18,7 @@ ERROR_NAMES = {-1: "MOC_ERR_ARG", -2: "MOC_ERR_RANGE", -3: "MOC_ERR_CYCLE", -4: 
                -5: "MOC_ERR_CUDA", -6: "MOC_ERR_NOMEM"}
 EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", "moc_graph_info",
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
-           "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc"]
+           "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -44,6 +44,8 @@ lib.moc_mem_profile.restype = ctypes.c_int
 lib.moc_mem_profile.argtypes = [_P, _P, _i32, _P, _P, _P, _P]
 lib.moc_graph_set_launch.restype = ctypes.c_int
 lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
+lib.moc_graph_set_timing_events.restype = ctypes.c_int
+lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
 lib.moc_last_launch_count.restype = ctypes.c_int
 lib.moc_last_launch_count.argtypes = []
 lib.moc_last_error.restype = ctypes.c_char_p
@@ -120,6 +122,18 @@ def moc_graph_set_max_copies(g, C):
 def moc_graph_set_launch(g, threads_per_sequence=0, sequences_per_block=0):
     _check(lib.moc_graph_set_launch(g, int(threads_per_sequence), int(sequences_per_block)),
            "moc_graph_set_launch")
+
+
+def moc_graph_set_timing_events(g, before=None, after=None):
+    """before/after: torch.cuda.Event(enable_timing=True) recorded around the evaluation kernel of
+    every following moc_eval_batch on this handle; None, None switches the hook off."""
+    def raw(ev):
+        if ev is None:
+            return None
+        if not ev.cuda_event:          # torch creates the CUDA event lazily, on the first record
+            ev.record()
+        return ctypes.c_void_p(ev.cuda_event)
+    _check(lib.moc_graph_set_timing_events(g, raw(before), raw(after)), "moc_graph_set_timing_events")
 
 
 def moc_graph_destroy(g):
@@ -218,6 +232,9 @@ class Graph:
 
     def info(self):
         return moc_graph_info(self.h)
+
+    def set_timing_events(self, before=None, after=None):
+        moc_graph_set_timing_events(self.h, before, after)
 
     def set_launch(self, threads_per_sequence=0, sequences_per_block=0):
         moc_graph_set_launch(self.h, threads_per_sequence, sequences_per_block)

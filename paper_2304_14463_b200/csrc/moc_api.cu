@@ -64,6 +64,7 @@ struct moc_graph {
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;
     int32_t want_G = 0, want_gpc = 0;
+    cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
     // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
     int32_t sell_len = 0, n_tiles = 0;
     void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
@@ -280,6 +281,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
     const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
     moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
     ++g_launches;
+    if (g->ev_before) MOC_CUDA(cudaEventRecord(g->ev_before, st));
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)pl.block);
@@ -323,6 +325,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
     }
     ++g_launches;
     MOC_CUDA(cudaGetLastError());
+    if (g->ev_after) MOC_CUDA(cudaEventRecord(g->ev_after, st));
     return MOC_OK;
 }
 
@@ -553,6 +556,15 @@ int moc_graph_set_launch(moc_graph* g, int32_t tps, int32_t spb) {
     g->want_G = tps;
     g->want_gpc = spb;
     g->plan_eval.valid = false;
+    return MOC_OK;
+}
+
+int moc_graph_set_timing_events(moc_graph* g, void* before, void* after) {
+    g_err[0] = 0;
+    if (!g || ((before == nullptr) != (after == nullptr)))
+        return fail(MOC_ERR_ARG, "moc_graph_set_timing_events: null handle, or only one of the two events given");
+    g->ev_before = (cudaEvent_t)before;
+    g->ev_after = (cudaEvent_t)after;
     return MOC_OK;
 }
 

@@ -218,6 +218,21 @@ def test_determinism_and_reuse(B):
     assert B.moc_last_launch_count() == 2
 
 
+def test_timing_hook(B):
+    wl = W.make(2, seed=8, B=2000)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    s, l = dev(wl.seqs), dev(wl.lens)
+    ref = [t.clone() for t in G.eval_batch(s, l, BIG)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    G.set_timing_events(e0, e1)
+    out = G.eval_batch(s, l, BIG)
+    G.set_timing_events(None, None)
+    torch.cuda.synchronize()
+    assert 0.0 < e0.elapsed_time(e1) < 50.0 and all(torch.equal(a, b) for a, b in zip(ref, out))
+    with pytest.raises(B.MocError):
+        B._check(B.lib.moc_graph_set_timing_events(G.h, None, 1), "half a pair")
+
+
 def test_host_entry_point(B):
     wl = W.make(1, seed=9, B=2000)
     O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
