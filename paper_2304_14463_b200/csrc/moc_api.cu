@@ -145,7 +145,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         const size_t v_max = ((nvec_d + 31) / 32) | 1;
         const size_t rec_b = (pl.wide ? sizeof(moc::NodeRec<int64_t>) : sizeof(moc::NodeRec<int32_t>)) * 64 * (size_t)g->n_tiles,
                      col_b = align16(4 * (size_t)g->n_tiles), jds_b = align16(4 * (size_t)g->sell_len),
-                     word_b = align16(4 * (n + 1)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
+                     word_b = align16(4 * (n + 2)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
         const size_t w_b = 8 * 64 * (size_t)g->n_tiles;
         const size_t graph_b = rec_b + w_b + col_b + jds_b, warp_b = word_b + moc::kPairWordTail + delta_b;
         PairFn fn = pl.wide ? (PairFn)moc::eval_pair_kernel<int64_t> : (PairFn)moc::eval_pair_kernel<int32_t>;
@@ -458,13 +458,14 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
             int64_t sell_len = 0;
             for (int32_t d = 0; d < n_tiles; ++d) {
                 for (int32_t s = 0; s < 64; ++s)
-                    if (slot[(size_t)d * 64 + s] >= 0) rows[d] = std::max(rows[d], deg(slot[(size_t)d * 64 + s]));
+                    if (slot[(size_t)d * 64 + s] >= 0)
+                        rows[d] = std::max(rows[d], std::max(1, deg(slot[(size_t)d * 64 + s])));  // a sink gets one entry
                 sell_len += 32 * (int64_t)rows[d];
             }
             int32_t max_rows = 0;
             for (int32_t d = 0; d < n_tiles; ++d) max_rows = std::max(max_rows, rows[d]);
             if (sell_len <= 2 * ne + 4096 && sell_len < (1 << 20) && max_rows < (1 << 12)) {
-                const uint32_t word_b = (uint32_t)align16(4 * ((size_t)n + 1));
+                const uint32_t word_b = (uint32_t)align16(4 * ((size_t)n + 2));
                 const uint32_t dummy = 4u * (uint32_t)n;
                 std::vector<uint32_t> tile((size_t)n_tiles);
                 std::vector<moc::NodeRec<int32_t>> rec32((size_t)n_halves * 32);
@@ -473,7 +474,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                 std::vector<uint32_t> sell((size_t)std::max<int64_t>(sell_len, 1), dummy | (dummy << 16));
                 for (size_t r = 0; r < slot.size(); ++r) {
                     const int32_t v = slot[r];
-                    const uint32_t nd = v >= 0 ? (4u * (uint32_t)v | ((uint32_t)deg(v) << 16)) : word_b;
+                    const uint32_t nd = v >= 0 ? 4u * (uint32_t)v : word_b;
                     rec32[r].nd = nd;
                     rec32[r].m = v >= 0 ? m32[v] : 0;
                     wslot[r] = v >= 0 ? w[v] : 0;
@@ -491,6 +492,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                             const int32_t v = slot[((size_t)2 * d + h) * 32 + l];
                             rem[l].clear();
                             if (v >= 0) rem[l].assign(succ.begin() + succ_start[v], succ.begin() + succ_start[v + 1]);
+                            if (v >= 0 && rem[l].empty()) rem[l].push_back(n + 1);  // sink: the word that holds T
                             lanes.push_back(l);
                         }
                         for (int32_t k = 0; k < rows[d]; ++k) {

@@ -2,33 +2,35 @@
 // C_v = 2, Section 4.3): one warp evaluates one sequence, warp-synchronously, with the graph staged
 // once per block in shared memory.
 //
-// Representation.  Positions are 1-based and 16 bits wide; 0 means "no copy".  Each node owns one
-// 32-bit word holding its (at most two) positions, so a consumer reads both copies of a
-// predecessor/successor with one load.  Lane l of a warp works on the nodes with id = l (mod 32):
-// a node's word then sits in bank l, so the lanes' reads of their own words never collide.  The
-// nodes of each residue class are sorted by out-degree (descending); "half" j holds the j-th node
-// of every class and a tile is two consecutive halves, so a lane treats two nodes per tile.  The
-// successor lists are stored per tile as a dense [rows][32] matrix of 32-bit entries: entry
-// (k, l) packs the word offsets of the k-th successor of lane l's two nodes, 16 bits each; rows =
-// largest out-degree in the tile; missing successors point at a dummy word that stays zero, which
-// is neutral for the maxima and minima taken over the successors.  Every lane of a warp runs the
-// same trip count.  Node slots beyond the last node of a class read a word that holds the
-// constant 1 and carry m = w = 0, so they need no special case.
+// Representation.  Positions are 1-based and 16 bits wide.  Each node owns one 32-bit word with
+// its two positions; a node computed once holds the same position in both halves, an absent node
+// holds 0.  A consumer reads both copies of a successor with one load.  Lane l of a warp works on
+// the nodes with id = l (mod 32): a node's word then sits in bank l, so the lanes' reads of their
+// own words never collide.  The nodes of each residue class are sorted by out-degree
+// (descending); "half" j holds the j-th node of every class and a tile is two consecutive halves,
+// so a lane treats two nodes per tile.  The successor lists are stored per tile as a dense
+// [rows][32] matrix of 32-bit entries: entry (k, l) packs the word offsets of the k-th successor
+// of lane l's two nodes, 16 bits each; rows = largest out-degree in the tile; missing successors
+// point at a dummy word that stays zero, which is neutral for every reduction below.  A sink has
+// one made-up successor: a word that holds the sequence length T, which keeps its last copy to
+// the end.  Every lane of a warp runs the same trip count.  Node slots beyond the last node of a
+// class read a constant word and carry m = w = 0, so they need no special case.
 //
 // Stages for one sequence seq[0..T) (paper: Section 2, Eqs. 1-8):
-//   1. occurrence words   step t exchanges t+1 into the low half of its node's word and moves the
-//                         previous occupant to the high half.  A third copy loses a position, which
-//                         the check "sum of stored positions == T(T+1)/2" detects; an absent node
-//                         (Eq. 7) shows as a zero low half.
+//   1. occurrence words   step t exchanges (t+1, t+1) into its node's word; if the word was taken,
+//                         the previous low half is stored into the high half.  An id outside
+//                         [0, n) lands in the dummy word.  A third copy, or an id out of range,
+//                         loses a position, which the check "sum of stored positions = T(T+1)/2"
+//                         detects; an absent node (Eq. 7) shows as a zero word.
 //   2. free steps         one lane per node u with copies a <= b (a = b if computed once), one pass
 //                         over its successors' words r with three packed 16-bit reductions:
-//                           F = max r            latest successor copy: b is kept until max(b, F);
-//                           D = min (r - 1)      earliest successor copy: before a = Eq. 5 violated;
+//                           F = max(b, r)        latest successor copy: b is kept until F;
+//                           D = min(a-1, r-1)    below a-1 iff a successor copy precedes a: Eq. 5
+//                                                violated;
 //                           G = max (r - b)      mod 2^16 this ranks the copies below b above all
 //                                                others, in order: the latest successor copy inside
 //                                                (a, b), until which the first copy a is kept
 //                                                (Eqs. 2, 3, 5).
-//                         A sink's last copy is kept to the end.
 //   3. memory profile     delta[p] += m_u, delta[free+1] -= m_u, prefix sum (Eq. 4).
 //   4. reductions         peak (Section 2), duration = sum_v w_v + sum over second copies (Eq. 1).
 #pragma once
@@ -44,7 +46,7 @@ struct PairParams {
     int32_t n_tiles;           // tiles of 64 node slots (two halves of 32)
     int32_t sell_len;          // 32-bit entries of the successor tiles
     int32_t max_T;             // C * n
-    uint32_t sum_bias;         // number of empty node slots (each reads a word holding 1)
+    uint32_t sum_bias;         // number of empty node slots (each reads a word holding (1, 1))
     const void* rec;           // 64 * n_tiles node records (NodeRec<MemT>), slot = half * 32 + lane
     const int64_t* wslot;      // 64 * n_tiles durations, same slots
     const uint32_t* sell;      // sell_len entries: successor word offsets of the two halves, 16 bits each
@@ -80,6 +82,12 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
     asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
+__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t swap_halves(uint32_t a) { return __byte_perm(a, 0, 0x1032); }
 
 // ---- shared-memory accesses by 32-bit shared address
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
@@ -102,7 +110,7 @@ __device__ __forceinline__ void red_add_shared(uint32_t addr, int64_t v) {
     asm volatile("red.shared.add.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 
-// Node record: byte offset of the node's word | out-degree << 16, and the output size.
+// Node record: byte offset of the node's word, and the output size.
 template <typename MemT> struct NodeRec;
 template <> struct __align__(8) NodeRec<int32_t> { uint32_t nd; int32_t m; };
 template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; int64_t m; };
@@ -134,7 +142,8 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     char* delta_base = ws + p.word_bytes + kPairWordTail;          // includes the front pad
     const uint32_t wa = (uint32_t)__cvta_generic_to_shared(word);
     const uint32_t da = (uint32_t)__cvta_generic_to_shared(delta_base) + kPairDeltaFront;  // &delta[0]
-    if (lane == 0) *reinterpret_cast<uint32_t*>(ws + p.word_bytes) = 1u;   // read by empty node slots
+    const uint32_t da1 = da - (uint32_t)sizeof(MemT);                                     // &delta[-1]
+    if (lane == 0) *reinterpret_cast<uint32_t*>(ws + p.word_bytes) = 0x00010001u;   // read by empty node slots
     __syncthreads();
 
     const int n = p.n;
@@ -169,6 +178,7 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 for (int i = lane; i < nd4; i += 32) d4[i] = z;
             }
             __syncwarp();
+            if (lane == 0) word[n + 1] = (uint32_t)T * 0x10001u;   // the made-up successor of sinks
 
             // ---- stage 1: occurrence words
             {
@@ -176,11 +186,10 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 const int a = (int)((reinterpret_cast<uintptr_t>(row) & 15) >> 2);
                 const int nvec = (T + a + 3) >> 2;
                 auto put = [&](int node, uint32_t t1) {
-                    if ((unsigned)node < (unsigned)n) {
-                        const uint32_t addr = wa + 4u * (uint32_t)node;
-                        const uint32_t old = exch_shared(addr, t1);
-                        if (old) sts_u16(addr + 2, old);
-                    }
+                    // ids outside [0, n) go to the dummy word n; the position sum exposes them
+                    const uint32_t addr = wa + 4u * min((uint32_t)node, (uint32_t)n);
+                    const uint32_t old = exch_shared(addr, t1 * 0x10001u);
+                    if (old) sts_u16(addr + 2, old);
                 };
                 // vectors that lie completely inside the row
                 for (int i = lane; i < nvec; i += 32) {
@@ -214,18 +223,17 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             int64_t dur_extra = 0;
             for (int d = 0; d < p.n_tiles; ++d) {
                 Rec rec[2];
-                uint32_t lo[2], hi[2], a[2], bpos[2], nbb[2], F[2], D[2], G[2];
+                uint32_t mn[2], mx[2], nbb[2], aa1[2], F[2], D[2], G[2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     rec[h] = s_rec[(2 * d + h) * 32 + lane];
-                    const uint32_t own = lds_u32(wa + (rec[h].nd & 0xFFFFu));
-                    lo[h] = own & 0xFFFFu;
-                    hi[h] = own >> 16;
-                    const uint32_t hh = hi[h] ? hi[h] : lo[h];
-                    a[h] = min(lo[h], hh);
-                    bpos[h] = max(lo[h], hh);
-                    nbb[h] = ((0u - bpos[h]) & 0xFFFFu) * 0x10001u;   // -b mod 2^16 in both halves
-                    F[h] = 0; D[h] = 0xFFFFFFFFu; G[h] = 0;
+                    const uint32_t own = lds_u32(wa + rec[h].nd);
+                    const uint32_t sw = swap_halves(own);
+                    mn[h] = min_u16x2(own, sw);        // (a, a)
+                    mx[h] = max_u16x2(own, sw);        // (b, b)
+                    nbb[h] = 0x00010000u - mx[h];      // (-b, -b) mod 2^16 for b >= 1
+                    aa1[h] = mn[h] - 0x00010001u;      // (a-1, a-1) for a >= 1
+                    F[h] = mx[h]; D[h] = aa1[h]; G[h] = 0;
                 }
                 // successors of the tile: uniform trip count, padded entries read the dummy word
                 const uint32_t tl = __shfl_sync(0xFFFFFFFFu, s_tile[d], 0);
@@ -245,22 +253,20 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 }
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint32_t deg = rec[h].nd >> 16;
-                    vmin = min(vmin, lo[h]);
-                    vsum += lo[h] + hi[h];
-                    const uint32_t Fm = max(F[h] & 0xFFFFu, F[h] >> 16);
-                    const uint32_t Dm = min(D[h] & 0xFFFFu, D[h] >> 16);
-                    // a successor copy before the first copy of u (deg = 0: D stays 0xFFFF)
-                    depw |= (Dm + 1 < a[h]) ? 1u : 0u;
-                    const uint32_t fb = deg != 0 ? max(Fm, bpos[h]) : (uint32_t)T;
-                    red_add_shared(da + ((bpos[h] - 1u) << kShift), rec[h].m);
+                    const uint32_t a = mn[h] & 0xFFFFu, bpos = mx[h] & 0xFFFFu;
+                    vmin = min(vmin, a);
+                    vsum += bpos;
+                    depw |= D[h] ^ aa1[h];     // some successor copy lies before the first copy of u
+                    const uint32_t fb = max_u16x2(F[h], swap_halves(F[h])) & 0xFFFFu;
+                    red_add_shared(da1 + (bpos << kShift), rec[h].m);
                     red_add_shared(da + (fb << kShift), (MemT)(-rec[h].m));
-                    if (hi[h] != 0) {
+                    if (a != bpos) {
+                        vsum += a;
                         dur_extra += s_w[(2 * d + h) * 32 + lane];
                         // latest successor copy x with a < x < b, if any: (x - b) mod 2^16 is the largest
-                        const uint32_t x = (max(G[h] & 0xFFFFu, G[h] >> 16) + bpos[h]) & 0xFFFFu;
-                        const uint32_t fa = (x - 1u < bpos[h] - 1u) ? x : a[h];
-                        red_add_shared(da + ((a[h] - 1u) << kShift), rec[h].m);
+                        const uint32_t x = (max_u16x2(G[h], swap_halves(G[h])) + bpos) & 0xFFFFu;
+                        const uint32_t fa = (x - 1u < bpos - 1u) ? x : a;
+                        red_add_shared(da1 + (a << kShift), rec[h].m);
                         red_add_shared(da + (fa << kShift), (MemT)(-rec[h].m));
                     }
                 }
