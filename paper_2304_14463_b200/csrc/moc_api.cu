@@ -274,13 +274,17 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     return p;
 }
 
-// Enqueues the offsets kernel and the evaluation kernel of plan `pl` with `offs` as scratch.
+// Enqueues the evaluation of plan `pl`.  With `offs` the offsets kernel runs first and the
+// evaluation kernel reads the packing offsets from that scratch; with offs == nullptr (only the
+// warp-per-sequence kernel can do that) the evaluation kernel finds the rows itself.
 int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_t* seqs, const int32_t* lens,
                  int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
                  cudaStream_t st) {
     const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
-    moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
-    ++g_launches;
+    if (offs) {
+        moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
+        ++g_launches;
+    }
     if (g->ev_before) MOC_CUDA(cudaEventRecord(g->ev_before, st));
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
@@ -329,6 +333,12 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_
     return MOC_OK;
 }
 
+// Each block of the self-addressing kernel re-reads the lengths in front of its range: worth it
+// while that redundant traffic (grid * B/2 * 4 bytes from L2) stays small next to a second launch.
+bool rows_without_scratch(const Plan& pl, int32_t B) {
+    return pl.pair && (int64_t)pl.grid * B * 2 <= (int64_t)16 << 20;
+}
+
 int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B, int64_t M,
                 int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st) {
     if (!g->plan_eval.valid) {
@@ -336,6 +346,8 @@ int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, in
         if (rc != MOC_OK) return rc;
     }
     const Plan& pl = g->plan_eval;
+    if (rows_without_scratch(pl, B))
+        return enqueue_eval(g, pl, nullptr, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
     int rc = ensure((void**)&g->d_offs, &g->offs_cap, ((size_t)B + 1) * sizeof(int64_t));
     if (rc != MOC_OK) return rc;
     if (pl.global_state) {

@@ -54,7 +54,7 @@ struct PairParams {
     int64_t base_dur;          // sum of all w
     const int32_t* seqs;
     const int32_t* lens;
-    const int64_t* offs;
+    const int64_t* offs;       // exclusive prefix sum of the lengths, or nullptr: the kernel finds the rows itself
     int32_t B;
     int64_t M;
     int64_t* out_peak;
@@ -118,6 +118,7 @@ template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; i
 template <typename MemT>
 __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     extern __shared__ __align__(16) char smem[];
+    __shared__ int64_t s_part[16];
     using Rec = NodeRec<MemT>;
     // ---- graph -> shared memory, once per block
     Rec* s_rec = reinterpret_cast<Rec*>(smem);
@@ -152,16 +153,63 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     constexpr int kShift = sizeof(MemT) == 4 ? 2 : 3;
     constexpr int kRegVecs = sizeof(MemT) == 4 ? 7 : 0;  // scan keeps up to this many vectors per lane in registers
 
-    int b = blockIdx.x * wpb + warp;
+    // Two ways to find the rows.  With p.offs (written by the offsets kernel) warps stride over the
+    // whole batch.  Without it (p.offs == nullptr) block c takes the contiguous range
+    // [c*B/grid, (c+1)*B/grid): it adds up the lengths in front of its range once, and every warp then
+    // walks the range with the lengths themselves -- no scratch, no second kernel.
+    const bool self = p.offs == nullptr;
+    int b, b_end, b_step;
     int64_t off = 0;
     int32_t T = 0;
-    if (b < p.B) { off = __ldg(&p.offs[b]); T = __ldg(&p.lens[b]); }
-    while (b < p.B) {
+    // self mode: lanes 0..wpb-1 hold the lengths of sequences b .. b+wpb-1 (next: of the following wpb)
+    int32_t len_raw = 0;
+    auto group_sum = [&](int32_t raw, int lanes) -> int64_t {   // sum of max(raw, 0) over lanes < `lanes`
+        const uint32_t v = (lane < lanes && raw > 0) ? (uint32_t)raw : 0u;
+        const uint32_t lo = __reduce_add_sync(0xFFFFFFFFu, v & 0xFFFFu), hi = __reduce_add_sync(0xFFFFFFFFu, v >> 16);
+        return (int64_t)lo + ((int64_t)hi << 16);
+    };
+    if (!self) {
+        b = blockIdx.x * wpb + warp;
+        b_end = p.B;
+        b_step = n_warps;
+        if (b < b_end) { off = __ldg(&p.offs[b]); T = __ldg(&p.lens[b]); }
+    } else {
+        const int c0 = (int)((int64_t)blockIdx.x * p.B / gridDim.x);
+        b_end = (int)(((int64_t)blockIdx.x + 1) * p.B / gridDim.x);
+        b_step = wpb;
+        int64_t sum = 0;
+        if ((reinterpret_cast<uintptr_t>(p.lens) & 15) == 0) {
+            const int4* l4 = reinterpret_cast<const int4*>(p.lens);
+            for (int i = threadIdx.x; i < (c0 >> 2); i += blockDim.x) {
+                const int4 q = __ldg(l4 + i);
+                sum += (int64_t)max(q.x, 0) + max(q.y, 0) + max(q.z, 0) + max(q.w, 0);
+            }
+            for (int i = (c0 & ~3) + threadIdx.x; i < c0; i += blockDim.x) sum += max(__ldg(p.lens + i), 0);
+        } else {
+            for (int i = threadIdx.x; i < c0; i += blockDim.x) sum += max(__ldg(p.lens + i), 0);
+        }
+        sum = warp_sum64(sum);
+        if (lane == 0) s_part[warp] = sum;
+        __syncthreads();
+        for (int k = 0; k < wpb; ++k) off += s_part[k];
+        // lengths of the first wpb sequences of the range; this warp starts at the warp-th of them
+        len_raw = (c0 + lane < p.B) ? __ldg(p.lens + c0 + lane) : 0;
+        off += group_sum(len_raw, warp);
+        b = c0 + warp;
+        // shift so that lane k holds the length of sequence b + k
+        len_raw = (b + lane < p.B) ? __ldg(p.lens + b + lane) : 0;
+        T = __shfl_sync(0xFFFFFFFFu, len_raw, 0);
+    }
+    while (b < b_end) {
         // fetch the next sequence's place early: its latency hides behind this sequence's work
-        const int b_next = b + n_warps;
+        const int b_next = b + b_step;
         int64_t off_next = 0;
-        int32_t T_next = 0;
-        if (b_next < p.B) { off_next = __ldg(&p.offs[b_next]); T_next = __ldg(&p.lens[b_next]); }
+        int32_t T_next = 0, len_next = 0;
+        if (!self) {
+            if (b_next < b_end) { off_next = __ldg(&p.offs[b_next]); T_next = __ldg(&p.lens[b_next]); }
+        } else {
+            if (b_next < b_end) len_next = (b_next + lane < p.B) ? __ldg(p.lens + b_next + lane) : 0;
+        }
 
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;
@@ -340,6 +388,11 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             p.out_peak[b] = out_pk;
             p.out_dur[b] = out_du;
             p.out_status[b] = out_st;
+        }
+        if (self) {
+            off_next = off + group_sum(len_raw, wpb);   // skip the wpb sequences b .. b+wpb-1
+            len_raw = len_next;
+            T_next = __shfl_sync(0xFFFFFFFFu, len_next, 0);
         }
         b = b_next;
         off = off_next;

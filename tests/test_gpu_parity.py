@@ -215,6 +215,9 @@ def test_determinism_and_reuse(B):
     # a smaller batch after a larger one on the same handle
     O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
     assert_batch_equal(G, O, wl.seqs[:int(wl.lens[:10].sum())], wl.lens[:10], BIG, "reuse")
+    assert B.moc_last_launch_count() == 1          # the warp-per-sequence kernel finds its rows itself
+    G.set_launch(64, 4)                            # the group kernel runs behind the offsets kernel
+    assert_batch_equal(G, O, wl.seqs[:int(wl.lens[:10].sum())], wl.lens[:10], BIG, "reuse, group kernel")
     assert B.moc_last_launch_count() == 2
 
 
