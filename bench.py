@@ -320,7 +320,7 @@ def main():
                          "kernel": "evaluation kernel (CUDA events around each launch, mean of %d)" % n_k,
                          "between_kernels_ms": float(np.mean(gap_ms)),
                          "note": "the kernel is bound by shared-memory wavefronts and instruction issue, "
-                                 "not by HBM (ALU pipe 63 %, shared-memory data pipe 60 %, DRAM 8 % in ncu)"},
+                                 "not by HBM (ncu: ALU pipe 52 %, shared-memory data pipe 59 %, DRAM 8 % busy)"},
             "clocks": clocks.summary(),
         }
         if not args.no_cpu_baseline:
