@@ -171,6 +171,34 @@ def test_unaligned_rows_and_views(B):
         assert (peak.cpu().numpy() == op).all() and (dur.cpu().numpy() == od).all() and (st.cpu().numpy() == os_).all()
 
 
+def test_rows_found_in_kernel(B):
+    """Batches small enough for the warp-per-sequence kernel to locate its rows itself: ranges that
+    do not divide evenly, fewer sequences than warps, a length array off a 16-byte boundary, very
+    long and negative lengths in front of valid rows."""
+    wl = W.make(2, seed=10, B=1500)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    rows = W.unpack(wl.seqs, wl.lens)
+    for nb in (1, 2, 11, 13, 445, 1499):
+        seqs, lens = W.pack(rows[:nb])
+        assert_batch_equal(G, O, seqs, lens, BIG, f"{nb} sequences")
+        assert B.moc_last_launch_count() == 1
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=6, frac=0.2)
+    lens = lens.copy()
+    junk = np.full(3000, 7, np.int32)
+    lens2 = np.concatenate([[-5, 3000], lens, [0, -1]]).astype(np.int32)     # a 3000-step malformed row first
+    seqs2 = np.concatenate([junk, seqs]).astype(np.int32)
+    op, od, os_, _ = O.eval_batch(seqs2, lens2, 10 ** 6)
+    buf = torch.zeros(len(lens2) + 3, dtype=torch.int32, device="cuda")
+    view = buf[1:1 + len(lens2)]
+    view.copy_(dev(lens2))
+    assert view.data_ptr() % 16 == 4
+    peak, dur, st = G.eval_batch(dev(seqs2), view, 10 ** 6)
+    torch.cuda.synchronize()
+    assert (peak.cpu().numpy() == op).all() and (dur.cpu().numpy() == od).all() and (st.cpu().numpy() == os_).all()
+    assert os_[0] == -2 and os_[1] == -2 and os_[-1] == -2
+
+
 def test_degenerate_batches(B):
     n = 5
     edges = [(0, 1), (1, 2), (0, 3)]
