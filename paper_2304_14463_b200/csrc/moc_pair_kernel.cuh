@@ -151,7 +151,6 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     const int n_warps = gridDim.x * wpb;
     constexpr int kPerVec = 16 / (int)sizeof(MemT);  // delta entries per 16-byte vector
     constexpr int kShift = sizeof(MemT) == 4 ? 2 : 3;
-    constexpr int kRegVecs = sizeof(MemT) == 4 ? 7 : 0;  // scan keeps up to this many vectors per lane in registers
 
     // Two ways to find the rows.  With p.offs (written by the offsets kernel) warps stride over the
     // whole batch.  Without it (p.offs == nullptr) block c takes the contiguous range
@@ -332,52 +331,37 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 out_du = p.base_dur + warp_sum64(dur_extra);
             } else {
                 // ---- stage 3 + 4: prefix sum and running maximum; lane owns V consecutive vectors
+                // One pass: the lane's running prefix and the largest prefix it sees; the largest
+                // usage inside the lane's chunk is then (sum of the chunks before it) + that maximum.
                 const int4* d4 = reinterpret_cast<const int4*>(delta_base + kPairDeltaFront) + lane * V;
-                MemT peak = 0;
-                if (kRegVecs > 0 && V <= kRegVecs) {
-                    int4 q[kRegVecs > 0 ? kRegVecs : 1];
-                    int32_t s = 0;
-#pragma unroll
-                    for (int j = 0; j < kRegVecs; ++j) {
-                        q[j] = make_int4(0, 0, 0, 0);
-                        if (j < V) q[j] = d4[j];
-                        s += q[j].x + q[j].y + q[j].z + q[j].w;
-                    }
-                    int32_t run = warp_inclusive_sum(s, lane) - s;
-                    int32_t pk = 0;
-#pragma unroll
-                    for (int j = 0; j < kRegVecs; ++j) {
-                        run += q[j].x; pk = max(pk, run);
-                        run += q[j].y; pk = max(pk, run);
-                        run += q[j].z; pk = max(pk, run);
-                        run += q[j].w; pk = max(pk, run);
-                    }
-                    peak = (MemT)pk;
-                } else {
-                    MemT s = 0;
-                    for (int j = 0; j < V; ++j) {
-                        const int4 q = d4[j];
-                        if constexpr (sizeof(MemT) == 4) s += q.x + q.y + q.z + q.w;
-                        else {
-                            const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
-                            s += (MemT)(l.x + l.y);
-                        }
-                    }
-                    MemT run = warp_inclusive_sum(s, lane) - s;
-                    for (int j = 0; j < V; ++j) {
-                        const int4 q = d4[j];
-                        if constexpr (sizeof(MemT) == 4) {
-                            run += q.x; peak = max(peak, run);
-                            run += q.y; peak = max(peak, run);
-                            run += q.z; peak = max(peak, run);
-                            run += q.w; peak = max(peak, run);
-                        } else {
-                            const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
-                            run += (MemT)l.x; peak = run > peak ? run : peak;
-                            run += (MemT)l.y; peak = run > peak ? run : peak;
-                        }
+                MemT run = 0, top;
+                {
+                    const int4 q = d4[0];
+                    if constexpr (sizeof(MemT) == 4) {
+                        run = q.x; top = run;
+                        run += q.y; top = max(top, run);
+                        run += q.z; top = max(top, run);
+                        run += q.w; top = max(top, run);
+                    } else {
+                        const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
+                        run = (MemT)l.x; top = run;
+                        run += (MemT)l.y; top = run > top ? run : top;
                     }
                 }
+                for (int j = 1; j < V; ++j) {
+                    const int4 q = d4[j];
+                    if constexpr (sizeof(MemT) == 4) {
+                        run += q.x; top = max(top, run);
+                        run += q.y; top = max(top, run);
+                        run += q.z; top = max(top, run);
+                        run += q.w; top = max(top, run);
+                    } else {
+                        const longlong2 l = *reinterpret_cast<const longlong2*>(&q);
+                        run += (MemT)l.x; top = run > top ? run : top;
+                        run += (MemT)l.y; top = run > top ? run : top;
+                    }
+                }
+                const MemT peak = warp_inclusive_sum(run, lane) - run + top;
                 out_pk = (int64_t)warp_max_t(peak);
                 out_du = p.base_dur + warp_sum64(dur_extra);
                 out_st = out_pk <= p.M ? 1 : 0;
