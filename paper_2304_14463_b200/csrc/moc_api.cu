@@ -120,13 +120,24 @@ KernelFn global_fn(int CP, bool profile) {
     }
 }
 
+// Raises a kernel's dynamic shared-memory limit to all the device offers beside its static part.
+cudaError_t raise_smem_limit(const void* fn, size_t smem_optin) {
+    cudaFuncAttributes a{};
+    cudaError_t e = cudaFuncGetAttributes(&a, fn);
+    if (e != cudaSuccess) return e;
+    const size_t room = smem_optin > a.sharedSizeBytes ? smem_optin - a.sharedSizeBytes : 0;
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)room);
+}
+
 int pow2_ceil(int x) {
     int p = 1;
     while (p < x) p <<= 1;
     return p;
 }
 
-// Chooses kernel variant, group size and grid for the handle's current n and C.
+// Chooses kernel variant, group size and grid for the handle's current n and C.  The dynamic
+// shared-memory limit of a kernel is a property of the kernel, not of the handle: it is always
+// raised to the device maximum, so that handles with different needs can share one kernel.
 int make_plan(const moc_graph* g, bool profile, Plan* out) {
     Plan pl;
     const int64_t n = g->n, C = g->C;
@@ -155,7 +166,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             const int wpb = g->want_gpc ? std::min(g->want_gpc, 16) : cand[ci];
             const size_t sm = graph_b + wpb * warp_b;
             if (sm > smem_cap) { if (g->want_gpc) break; else continue; }
-            if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
             int nb = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, wpb * 32, sm) != cudaSuccess) { cudaGetLastError(); continue; }
             if (nb * wpb > best_warps) { best_warps = nb * wpb; best_wpb = wpb; best_nb = nb; }
@@ -171,7 +182,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             pl.grid = g->sm_count * best_nb;
             pl.rec_bytes = (uint32_t)rec_b; pl.w_bytes = (uint32_t)w_b; pl.tile_bytes = (uint32_t)col_b;
             pl.sell_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
-            cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+            cudaError_t e = raise_smem_limit((const void*)fn, g->smem_optin);
             if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
             pl.valid = true;
             *out = pl;
@@ -199,7 +210,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         pl.smem = (size_t)gpc * sh_group;
         pl.fn = pl.wide ? shared_fn_g<int64_t>(G, pl.CP, profile) : shared_fn_g<int32_t>(G, pl.CP, profile);
         if (!pl.fn) return fail(MOC_ERR_ARG, "unsupported launch shape");
-        cudaError_t e = cudaFuncSetAttribute((const void*)pl.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+        cudaError_t e = raise_smem_limit((const void*)pl.fn, g->smem_optin);
         if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         int nb = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)pl.fn, pl.block, pl.smem);

@@ -249,6 +249,20 @@ def test_determinism_and_reuse(B):
     assert B.moc_last_launch_count() == 2
 
 
+def test_handles_of_different_size_interleaved(B):
+    """Two graphs that use the same kernels with very different shared-memory footprints."""
+    big = W.make(2, seed=11, B=600)
+    small = W.make(0, seed=11, B=600)
+    Gb, Gs = B.Graph(big.n, big.edges, big.w, big.m, big.C), B.Graph(small.n, small.edges, small.w, small.m, small.C)
+    Ob, Os = OracleGraph(big.n, big.edges, big.w, big.m, big.C), OracleGraph(small.n, small.edges, small.w, small.m, small.C)
+    for shape in ((0, 0), (128, 2)):
+        Gb.set_launch(*shape)
+        Gs.set_launch(*shape)
+        for _ in range(2):
+            assert_batch_equal(Gb, Ob, big.seqs, big.lens, BIG, "large graph")
+            assert_batch_equal(Gs, Os, small.seqs, small.lens, BIG, "small graph")
+
+
 def test_timing_hook(B):
     wl = W.make(2, seed=8, B=2000)
     G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
