@@ -120,6 +120,19 @@ KernelFn global_fn(int CP, bool profile) {
     }
 }
 
+template <typename MemT>
+PairFn pair_fn_t(int pre) {
+    switch (pre) {
+        case 0: return (PairFn)moc::eval_pair_kernel<MemT, 0>;
+        case 1: return (PairFn)moc::eval_pair_kernel<MemT, 1>;
+        case 2: return (PairFn)moc::eval_pair_kernel<MemT, 2>;
+        case 3: return (PairFn)moc::eval_pair_kernel<MemT, 3>;
+        case 4: return (PairFn)moc::eval_pair_kernel<MemT, 4>;
+        default: return (PairFn)moc::eval_pair_kernel<MemT, 5>;
+    }
+}
+PairFn pair_fn(bool wide, int pre) { return wide ? pair_fn_t<int64_t>(pre) : pair_fn_t<int32_t>(pre); }
+
 // Raises a kernel's dynamic shared-memory limit to all the device offers beside its static part.
 cudaError_t raise_smem_limit(const void* fn, size_t smem_optin) {
     cudaFuncAttributes a{};
@@ -159,7 +172,9 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
                      word_b = align16(4 * (n + 2)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
         const size_t w_b = 8 * 64 * (size_t)g->n_tiles;
         const size_t graph_b = rec_b + w_b + col_b + jds_b, warp_b = word_b + moc::kPairWordTail + delta_b;
-        PairFn fn = pl.wide ? (PairFn)moc::eval_pair_kernel<int64_t> : (PairFn)moc::eval_pair_kernel<int32_t>;
+        // vectors of the next row fetched ahead per lane: enough for a typical row of about 1.3 n steps
+        const int pre = n < 256 ? 0 : (int)std::min<int64_t>(5, (n * 13 / 10 + 96) / 128);
+        PairFn fn = pair_fn(pl.wide, pre);
         int best_wpb = 0, best_warps = 0, best_nb = 0;
         const int cand[4] = {16, 12, 8, 4};
         for (int ci = 0; ci < 4; ++ci) {

@@ -115,7 +115,9 @@ template <typename MemT> struct NodeRec;
 template <> struct __align__(8) NodeRec<int32_t> { uint32_t nd; int32_t m; };
 template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; int64_t m; };
 
-template <typename MemT>
+// kPre: how many 16-byte vectors of the next row each lane fetches ahead (rows of about 128*kPre
+// steps; 0 for short rows, where the extra registers cost more than the wait)
+template <typename MemT, int kPre>
 __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
     extern __shared__ __align__(16) char smem[];
     __shared__ int64_t s_part[16];
@@ -199,6 +201,10 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
         len_raw = (b + lane < p.B) ? __ldg(p.lens + b + lane) : 0;
         T = __shfl_sync(0xFFFFFFFFu, len_raw, 0);
     }
+    // The first kPre 16-byte vectors per lane of the NEXT row are loaded into registers while the
+    // current sequence is still being worked on, so that stage 1 does not wait for HBM.
+    int4 pre[kPre > 0 ? kPre : 1];
+    bool have_pre = false;
     while (b < b_end) {
         // fetch the next sequence's place early: its latency hides behind this sequence's work
         const int b_next = b + b_step;
@@ -210,6 +216,8 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
             if (b_next < b_end) len_next = (b_next + lane < p.B) ? __ldg(p.lens + b_next + lane) : 0;
         }
 
+        const bool use_pre = have_pre;   // pre[] holds this row only if the previous iteration fetched it
+        have_pre = false;
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;
         if (T >= n && T <= p.max_T) {
@@ -238,8 +246,21 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                     const uint32_t old = exch_shared(addr, t1 * 0x10001u);
                     if (old) sts_u16(addr + 2, old);
                 };
-                // vectors that lie completely inside the row
-                for (int i = lane; i < nvec; i += 32) {
+                // vectors that lie completely inside the row (the first kPre per lane may already be here)
+#pragma unroll
+                for (int j = 0; j < kPre; ++j) {
+                    const int i = lane + 32 * j;
+                    const int t0 = 4 * i - a;
+                    if (i < nvec && t0 >= 0 && t0 + 4 <= T) {
+                        int4 v = pre[j];
+                        if (!use_pre) v = __ldg(reinterpret_cast<const int4*>(row + t0));
+                        put(v.x, (uint32_t)t0 + 1);
+                        put(v.y, (uint32_t)t0 + 2);
+                        put(v.z, (uint32_t)t0 + 3);
+                        put(v.w, (uint32_t)t0 + 4);
+                    }
+                }
+                for (int i = lane + 32 * kPre; i < nvec; i += 32) {
                     const int t0 = 4 * i - a;
                     if (t0 >= 0 && t0 + 4 <= T) {
                         const int4 v = __ldg(reinterpret_cast<const int4*>(row + t0));
@@ -263,6 +284,24 @@ __global__ void __launch_bounds__(512) eval_pair_kernel(const PairParams p) {
                 }
             }
             __syncwarp();
+
+            // request the next row now: the loads complete behind stages 2-4
+            if (kPre > 0 && b_next < b_end) {
+                const int64_t off_n = self ? off + group_sum(len_raw, wpb) : off_next;
+                const int32_t T_n = self ? __shfl_sync(0xFFFFFFFFu, len_next, 0) : T_next;
+                if (T_n >= n && T_n <= p.max_T) {
+                    const int32_t* nrow = p.seqs + off_n;
+                    const int an = (int)((reinterpret_cast<uintptr_t>(nrow) & 15) >> 2);
+                    const int nvn = (T_n + an + 3) >> 2;
+#pragma unroll
+                    for (int j = 0; j < kPre; ++j) {
+                        const int i = lane + 32 * j;
+                        const int t0 = 4 * i - an;
+                        if (i < nvn && t0 >= 0 && t0 + 4 <= T_n) pre[j] = __ldg(reinterpret_cast<const int4*>(nrow + t0));
+                    }
+                    have_pre = true;
+                }
+            }
 
             // ---- stage 2 and the scatter of stage 3: two node slots per lane and tile
             uint32_t vmin = 0xFFFFFFFFu, vsum = 0;
