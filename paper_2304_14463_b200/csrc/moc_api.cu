@@ -177,8 +177,9 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         PairFn fn = pair_fn(pl.wide, pre);
         int best_wpb = 0, best_warps = 0, best_nb = 0;
         const int cand[4] = {16, 12, 8, 4};
+        const int max_wpb = pre > 0 ? 12 : 16;   // the look-ahead variants are compiled for at most 384 threads
         for (int ci = 0; ci < 4; ++ci) {
-            const int wpb = g->want_gpc ? std::min(g->want_gpc, 16) : cand[ci];
+            const int wpb = std::min(g->want_gpc ? g->want_gpc : cand[ci], max_wpb);
             const size_t sm = graph_b + wpb * warp_b;
             if (sm > smem_cap) { if (g->want_gpc) break; else continue; }
             if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
