@@ -15,16 +15,19 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "moc_oracle.c")
+_SRC_SEARCH = os.path.join(_HERE, "moc_search_oracle.c")
 _LIB = os.path.join(_HERE, "libmoc_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
-    """Compiles moc_oracle.c into libmoc_oracle.so next to it (gcc -O2); returns the path."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    """Compiles moc_oracle.c and moc_search_oracle.c into libmoc_oracle.so next to them (gcc -O2);
+    returns the path."""
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_SEARCH))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".{os.getpid()}.tmp"
-        subprocess.run(["gcc", "-O2", "-std=c11", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC],
-                       check=True)
+        subprocess.run(["gcc", "-O2", "-std=c11", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC,
+                        _SRC_SEARCH], check=True)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -42,6 +45,18 @@ def load_library(path):
     lib.moc_oracle_eval_batch.restype = ctypes.c_int32
     lib.moc_oracle_eval_batch.argtypes = [P, P, P, ctypes.c_int64, ctypes.c_int64, P, P, P,
                                           ctypes.c_int32]
+    if hasattr(lib, "moc_oracle_search_run"):
+        u32, u64, i32, i64 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_int64
+        lib.moc_oracle_philox4x32_10.restype = None
+        lib.moc_oracle_philox4x32_10.argtypes = [P, P, P]
+        lib.moc_oracle_mutate.restype = i32
+        lib.moc_oracle_mutate.argtypes = [P, i32, u32, u32, u32, P]
+        lib.moc_oracle_accept.restype = i32
+        lib.moc_oracle_accept.argtypes = [i64, i64, i32, i64, i64, i32, i64]
+        lib.moc_oracle_search_run.restype = None
+        lib.moc_oracle_search_run.argtypes = [P, P, P, P, P, P, i32, i32, i64, u64, u32, u32, P]
+        lib.moc_oracle_search_best.restype = i32
+        lib.moc_oracle_search_best.argtypes = [P, P, P, i32, i64]
     return lib
 
 
@@ -103,3 +118,69 @@ class OracleGraph:
         used = self._lib.moc_oracle_eval_batch(self._h, _ptr(seqs), _ptr(lens), B, int(M), _ptr(peak),
                                              _ptr(dur), _ptr(status), int(n_threads))
         return peak, dur, status, int(used)
+
+
+# ---- local search over sequences (moc_search_oracle.c) ----------------------------------------------
+
+def philox4x32_10(ctr, key, lib=None):
+    """One block of Philox4x32-10: ctr = 4 uint32, key = 2 uint32 -> 4 uint32."""
+    lib = lib if lib is not None else _load()
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, np.uint32)
+    lib.moc_oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def mutate(seq, r0, r1, r2, lib=None):
+    """The proposal the draws (r0, r1, r2) make from ``seq``; None for an empty sequence."""
+    lib = lib if lib is not None else _load()
+    seq = np.ascontiguousarray(seq, dtype=np.int32)
+    child = np.zeros(len(seq) + 2, np.int32)
+    Tc = lib.moc_oracle_mutate(_ptr(seq), len(seq), int(r0), int(r1), int(r2), _ptr(child))
+    return None if Tc < 0 else child[:Tc].copy()
+
+
+def accept(child, parent, M, lib=None):
+    """child, parent = (peak, dur, status) -> bool: the proposal replaces the chain's sequence."""
+    lib = lib if lib is not None else _load()
+    return bool(lib.moc_oracle_accept(int(child[0]), int(child[1]), int(child[2]), int(parent[0]),
+                                      int(parent[1]), int(parent[2]), int(M)))
+
+
+class OracleSearch:
+    """P chains of the search: rows of ``stride`` ints with lengths and evaluations."""
+
+    def __init__(self, graph: OracleGraph, seqs, lens, M, seed, stride=None):
+        self.g = graph
+        self._lib = graph._lib
+        self.M = int(M)
+        self.seed = int(seed)
+        lens = np.ascontiguousarray(lens, dtype=np.int32)
+        self.P = len(lens)
+        self.stride = int(stride) if stride is not None else graph.C * graph.n
+        self.pop = np.zeros((self.P, self.stride), np.int32)
+        offs = np.concatenate([[0], np.cumsum(np.clip(lens, 0, None))])
+        for c in range(self.P):
+            assert lens[c] <= self.stride
+            self.pop[c, :max(lens[c], 0)] = seqs[offs[c]:offs[c + 1]]
+        self.lens = np.clip(lens, 0, None).astype(np.int32)
+        self.peak, self.dur, self.status, _ = graph.eval_batch(seqs, lens, self.M)
+        self.generation = 0
+        self.accepted = 0
+
+    def run(self, n_gen):
+        acc = np.zeros(1, np.int64)
+        self._lib.moc_oracle_search_run(self.g._h, _ptr(self.pop), _ptr(self.lens), _ptr(self.peak),
+                                        _ptr(self.dur), _ptr(self.status), self.P, self.stride, self.M,
+                                        self.seed, self.generation, int(n_gen), _ptr(acc))
+        self.generation += int(n_gen)
+        self.accepted += int(acc[0])
+        return int(acc[0])
+
+    def best(self):
+        return int(self._lib.moc_oracle_search_best(_ptr(self.peak), _ptr(self.dur), _ptr(self.status),
+                                                    self.P, self.M))
+
+    def row(self, c):
+        return self.pop[c, :self.lens[c]].copy()
