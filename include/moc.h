@@ -160,6 +160,83 @@ int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t
                     int32_t* out_free, int32_t* out_status, void* stream);
 
 /*
+ * ---- Local search over sequences (Section 3, "Optimization in Two Phases") -------------------------
+ *
+ * P independent chains each hold one sequence and its evaluation.  One generation proposes, for
+ * every chain, one edited copy of its sequence, evaluates all proposals as one batch with the
+ * evaluator above, and replaces a chain's sequence by its proposal when the proposal's status is
+ * >= 0 and its key
+ *         ( max(peak, M), duration )                 (sequences with status < 0 rank last)
+ * is not larger than the chain's.  This folds the paper's two phases into one order: while a chain
+ * is over the budget the first component, the Phase 1 objective max(M_var, M), goes down; once
+ * peak <= M it equals M for everything that can still be accepted, so the duration (Eq. 1) alone
+ * decides under the memory constraint of Eq. 4, which is Phase 2.  Equal keys are accepted, so a
+ * chain can drift across plateaus.
+ *
+ * Proposal of chain c in generation k for a sequence of T steps (T = 0 proposes nothing): with
+ * (r0, r1, r2, r3) = Philox4x32-10(counter = (k, c, 0, 0), key = (seed mod 2^32, seed div 2^32))
+ * (Salmon, Moraes, Dror, Shaw, SC 2011),
+ *     op = r0 mod 3, q = r1 mod T;
+ *     op 0  insert: a further copy of node seq[q] is put in front of index j = r2 mod (T+1);
+ *     op 1  delete: element q is removed;
+ *     op 2  move:   element q is removed and put back in front of index j = r2 mod T of the
+ *                   shortened sequence.
+ * Whether a proposal is admissible is left to the evaluator (length outside [n, C*n], a node without
+ * a copy or with more than C copies give status -2; a consumer moved in front of its producer gives
+ * status -1), and such proposals are refused.
+ *
+ * The handle owns all device memory of the search (2 rows of C*n ints per chain plus 60 bytes per
+ * chain) and refers to the graph handle, which must outlive it and keep its C.  Calls on one search
+ * handle, and calls on its graph handle, must be ordered like calls on a graph handle.
+ */
+typedef struct moc_search moc_search; /* opaque */
+
+/*
+ * Starts a search from P sequences.
+ *   seqs, lens   DEVICE, packed as for moc_eval_batch; every length must lie in [0, C*n]
+ *                (MOC_ERR_ARG otherwise).  Sequences may be invalid (status < 0): such a chain
+ *                accepts the first proposal with status >= 0.
+ *   M            memory budget;  seed: key of the random draws.
+ * Copies the sequences, evaluates them and synchronises `stream` before returning.
+ * Errors: MOC_ERR_ARG, MOC_ERR_CUDA, MOC_ERR_NOMEM; *out is NULL on error.
+ */
+int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t P,
+                      int64_t M, uint64_t seed, void* stream, moc_search** out);
+
+/* Enqueues n_generations further generations on `stream` (asynchronous; two kernels per generation
+ * plus one at the end, no allocation, no synchronisation).  Generations are numbered from 0 over
+ * the life of the handle; the result does not depend on how they are split over calls. */
+int moc_search_run(moc_search* s, int32_t n_generations, void* stream);
+
+/*
+ * Copies the chains' current state to DEVICE arrays of the caller (any pointer may be NULL):
+ *   out_rows      P rows of `stride` ints (moc_search_info); row c holds chain c's sequence in its
+ *                 first out_lens[c] entries, the rest of the row is left untouched;
+ *   out_lens, out_status, out_accepted   P int32 (accepted = proposals accepted so far);
+ *   out_peak, out_dur                    P int64.
+ * Asynchronous on `stream`.
+ */
+int moc_search_state(const moc_search* s, int32_t* out_rows, int32_t* out_lens, int64_t* out_peak,
+                     int64_t* out_dur, int32_t* out_status, int32_t* out_accepted, void* stream);
+
+/*
+ * Best chain: smallest key among the chains with status >= 0, lowest index among equals.
+ *   out_seq    DEVICE, C*n ints, receives its sequence; may be NULL.
+ *   out_best   DEVICE, 6 int64: chain index (-1 when no chain is valid; the next four are then
+ *              0, -1, -1, -2), length, peak, duration, status, and the number of proposals
+ *              accepted so far over all chains.
+ * Asynchronous on `stream`.
+ */
+int moc_search_best(const moc_search* s, int32_t* out_seq, int64_t* out_best, void* stream);
+
+/* Facts about a search handle (any pointer may be NULL): number of chains, ints per exported row,
+ * generations enqueued so far. */
+int moc_search_info(const moc_search* s, int32_t* P, int32_t* stride, uint32_t* generation);
+
+/* Frees the handle and its device memory; NULL is accepted.  Synchronise its streams first. */
+void moc_search_destroy(moc_search* s);
+
+/*
  * Launch shape override for moc_eval_batch, for tuning.  threads_per_sequence is the number of
  * threads that cooperate on one sequence (32, 64, 128, 256, 512 or 1024; 0 = choose from the
  * graph size), sequences_per_block how many sequences one thread block works on at a time
@@ -176,7 +253,8 @@ int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t seq
  */
 int moc_graph_set_timing_events(moc_graph* g, void* before, void* after);
 
-/* Number of kernels the most recent moc_eval_batch / moc_mem_profile on this thread launched. */
+/* Number of kernels the most recent moc_eval_batch / moc_mem_profile / moc_search_run on this
+ * thread launched. */
 int moc_last_launch_count(void);
 
 /* Text of the most recent error on the calling thread ("" if none). Owned by the library. */

@@ -18,7 +18,9 @@ ERROR_NAMES = {-1: "MOC_ERR_ARG", -2: "MOC_ERR_RANGE", -3: "MOC_ERR_CYCLE", -4: 
                -5: "MOC_ERR_CUDA", -6: "MOC_ERR_NOMEM"}
 EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", "moc_graph_info",
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
-           "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events"]
+           "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
+           "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
+           "moc_search_destroy"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -46,6 +48,18 @@ lib.moc_graph_set_launch.restype = ctypes.c_int
 lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
 lib.moc_graph_set_timing_events.restype = ctypes.c_int
 lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
+lib.moc_search_create.restype = ctypes.c_int
+lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, _P, ctypes.POINTER(_P)]
+lib.moc_search_run.restype = ctypes.c_int
+lib.moc_search_run.argtypes = [_P, _i32, _P]
+lib.moc_search_state.restype = ctypes.c_int
+lib.moc_search_state.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P]
+lib.moc_search_best.restype = ctypes.c_int
+lib.moc_search_best.argtypes = [_P, _P, _P, _P]
+lib.moc_search_info.restype = ctypes.c_int
+lib.moc_search_info.argtypes = [_P, _P, _P, _P]
+lib.moc_search_destroy.restype = None
+lib.moc_search_destroy.argtypes = [_P]
 lib.moc_last_launch_count.restype = ctypes.c_int
 lib.moc_last_launch_count.argtypes = []
 lib.moc_last_error.restype = ctypes.c_char_p
@@ -209,6 +223,59 @@ def moc_last_launch_count():
     return lib.moc_last_launch_count()
 
 
+def moc_search_create(g, seqs, lens, M, seed):
+    """Device tensors (packed sequences, lengths) -> search handle; synchronous."""
+    import torch
+    h = _P()
+    rc = lib.moc_search_create(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"), lens.numel(),
+                               int(M), ctypes.c_uint64(int(seed)), _stream(), ctypes.byref(h))
+    _check(rc, "moc_search_create")
+    return h
+
+
+def moc_search_run(s, n_generations):
+    _check(lib.moc_search_run(s, int(n_generations), _stream()), "moc_search_run")
+
+
+def moc_search_info(s):
+    P, stride, gen = _i32(), _i32(), ctypes.c_uint32()
+    _check(lib.moc_search_info(s, ctypes.byref(P), ctypes.byref(stride), ctypes.byref(gen)), "moc_search_info")
+    return dict(P=P.value, stride=stride.value, generation=gen.value)
+
+
+def moc_search_state(s, want_rows=True):
+    """-> dict of device tensors: rows [P, stride] (or None), lens, peak, dur, status, accepted."""
+    import torch
+    info = moc_search_info(s)
+    P = info["P"]
+    rows = torch.zeros((P, info["stride"]), dtype=torch.int32, device="cuda") if want_rows else None
+    lens = torch.empty(P, dtype=torch.int32, device="cuda")
+    peak = torch.empty(P, dtype=torch.int64, device="cuda")
+    dur = torch.empty(P, dtype=torch.int64, device="cuda")
+    status = torch.empty(P, dtype=torch.int32, device="cuda")
+    acc = torch.empty(P, dtype=torch.int32, device="cuda")
+    rc = lib.moc_search_state(s, ctypes.c_void_p(rows.data_ptr()) if want_rows else None,
+                              ctypes.c_void_p(lens.data_ptr()), ctypes.c_void_p(peak.data_ptr()),
+                              ctypes.c_void_p(dur.data_ptr()), ctypes.c_void_p(status.data_ptr()),
+                              ctypes.c_void_p(acc.data_ptr()), _stream())
+    _check(rc, "moc_search_state")
+    return dict(rows=rows, lens=lens, peak=peak, dur=dur, status=status, accepted=acc)
+
+
+def moc_search_best(s, max_len):
+    """-> (seq tensor of max_len ints on the device, out_best tensor of 6 int64 on the device)."""
+    import torch
+    seq = torch.zeros(max_len, dtype=torch.int32, device="cuda")
+    best = torch.empty(6, dtype=torch.int64, device="cuda")
+    _check(lib.moc_search_best(s, ctypes.c_void_p(seq.data_ptr()), ctypes.c_void_p(best.data_ptr()), _stream()),
+           "moc_search_best")
+    return seq, best
+
+
+def moc_search_destroy(s):
+    lib.moc_search_destroy(s)
+
+
 class Graph:
     """Owns a moc_graph handle (created on the current CUDA device)."""
 
@@ -259,3 +326,37 @@ class Graph:
         if int(st[0]) != 1:
             raise ValueError("identity order is not a topological order of this graph")
         return int(peak[0])
+
+
+class Search:
+    """Owns a moc_search handle; keeps its Graph alive."""
+
+    def __init__(self, graph: Graph, seqs, lens, M, seed):
+        self.graph = graph
+        self.M = int(M)
+        self.h = moc_search_create(graph.h, seqs, lens, M, seed)
+
+    def close(self, _destroy=lib.moc_search_destroy):
+        if getattr(self, "h", None):
+            _destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def run(self, n_generations):
+        moc_search_run(self.h, n_generations)
+
+    def info(self):
+        return moc_search_info(self.h)
+
+    def state(self, want_rows=True):
+        return moc_search_state(self.h, want_rows)
+
+    def best(self):
+        """-> dict(index, seq (numpy), peak, dur, status, accepted); synchronises."""
+        import torch
+        seq, b = moc_search_best(self.h, self.graph.C * self.graph.n)
+        torch.cuda.synchronize()
+        b = b.cpu().numpy()
+        return dict(index=int(b[0]), seq=seq[:int(b[1])].cpu().numpy(), peak=int(b[2]), dur=int(b[3]),
+                    status=int(b[4]), accepted=int(b[5]))

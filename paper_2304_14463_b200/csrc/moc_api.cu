@@ -7,15 +7,17 @@
 #include <new>
 #include <vector>
 
-#include "../../include/moc.h"
-#include "moc_kernels.cuh"
-#include "moc_pair_kernel.cuh"
+#include "moc_host.cuh"
+
+using namespace moc_host;
 
 namespace {
-
 thread_local char g_err[512] = "";
-thread_local int g_launches = 0;
+thread_local int g_launches_tl = 0;
+}  // namespace
+#define g_launches (moc_host::launch_counter())
 
+namespace moc_host {
 int fail(int code, const char* fmt, ...) {
     va_list ap;
     va_start(ap, fmt);
@@ -23,66 +25,9 @@ int fail(int code, const char* fmt, ...) {
     va_end(ap);
     return code;
 }
-
-#define MOC_CUDA(call)                                                                      \
-    do {                                                                                    \
-        cudaError_t e_ = (call);                                                            \
-        if (e_ != cudaSuccess)                                                              \
-            return fail(e_ == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA,     \
-                        "%s: %s", #call, cudaGetErrorString(e_));                           \
-    } while (0)
-
-using KernelFn = void (*)(const moc::EvalParams);
-using PairFn = void (*)(const moc::PairParams);
-
-struct Plan {
-    bool valid = false;
-    KernelFn fn = nullptr;
-    int G = 0, gpc = 0, grid = 0, block = 0, CP = 0;
-    size_t smem = 0;
-    bool global_state = false, wide = false;
-    uint32_t cnt_bytes = 0, occ_bytes = 0, delta_bytes = 0, group_bytes = 0;
-    // fast path for C <= 2: a warp per sequence, graph staged in shared memory
-    bool pair = false;
-    PairFn pair_fn = nullptr;
-    uint32_t rec_bytes = 0, w_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
-};
-
-}  // namespace
-
-struct moc_graph {
-    int32_t n = 0;
-    int64_t n_edges = 0;  // distinct
-    int32_t C = 2;
-    int device = 0;
-    int sm_count = 0;
-    size_t smem_optin = 0;
-    int64_t sum_m = 0, sum_w = 0;
-    int32_t* d_succ_start = nullptr;
-    int32_t* d_succ = nullptr;
-    int64_t* d_w = nullptr;
-    int64_t* d_m64 = nullptr;
-    int32_t* d_m32 = nullptr;
-    int32_t want_G = 0, want_gpc = 0;
-    cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
-    // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
-    int32_t sell_len = 0, n_tiles = 0;
-    void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
-    void* d_rec64 = nullptr;
-    int64_t* d_wslot = nullptr;
-    uint32_t* d_sell = nullptr;
-    uint32_t* d_tile = nullptr;
-    // grow-only scratch; mutable because evaluation takes a const handle
-    mutable Plan plan_eval, plan_profile;
-    mutable int64_t* d_offs = nullptr;
-    mutable size_t offs_cap = 0;
-    mutable char* d_state = nullptr;
-    mutable size_t state_cap = 0;
-    mutable int32_t* d_stage_seqs = nullptr;
-    mutable size_t stage_seqs_cap = 0;
-    mutable char* d_stage_io = nullptr;  // lens | peak | dur | status
-    mutable size_t stage_io_cap = 0;
-};
+void clear_error() { g_err[0] = 0; }
+int& launch_counter() { return g_launches_tl; }
+}  // namespace moc_host
 
 namespace {
 
@@ -273,19 +218,6 @@ int ensure(void** ptr, size_t* cap, size_t need) {
     return MOC_OK;
 }
 
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = false;
-    explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) != cudaSuccess) return;
-        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
-    }
-    ~DeviceGuard() {
-        int cur = -1;
-        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
-    }
-};
-
 moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     moc::EvalParams p{};
     p.g.n = g->n;
@@ -301,14 +233,15 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     return p;
 }
 
-// Enqueues the evaluation of plan `pl`.  With `offs` the offsets kernel runs first and the
-// evaluation kernel reads the packing offsets from that scratch; with offs == nullptr (only the
-// warp-per-sequence kernel can do that) the evaluation kernel finds the rows itself.
-int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, const int32_t* seqs, const int32_t* lens,
+// Enqueues the evaluation of plan `pl`.  With `offs` the evaluation kernel reads the row offsets
+// from that array, which the offsets kernel fills first from the lengths when `fill_offs` is set
+// (packed rows) and which the caller has filled otherwise; with offs == nullptr (only the
+// warp-per-sequence kernel can do that) the evaluation kernel finds the packed rows itself.
+int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_offs, const int32_t* seqs, const int32_t* lens,
                  int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
                  cudaStream_t st) {
     const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
-    if (offs) {
+    if (offs && fill_offs) {
         moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
         ++g_launches;
     }
@@ -374,17 +307,33 @@ int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, in
     }
     const Plan& pl = g->plan_eval;
     if (rows_without_scratch(pl, B))
-        return enqueue_eval(g, pl, nullptr, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
+        return enqueue_eval(g, pl, nullptr, false, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
     int rc = ensure((void**)&g->d_offs, &g->offs_cap, ((size_t)B + 1) * sizeof(int64_t));
     if (rc != MOC_OK) return rc;
     if (pl.global_state) {
         rc = ensure((void**)&g->d_state, &g->state_cap, (size_t)pl.grid * pl.group_bytes);
         if (rc != MOC_OK) return rc;
     }
-    return enqueue_eval(g, pl, g->d_offs, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
+    return enqueue_eval(g, pl, g->d_offs, true, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
 }
 
 }  // namespace
+
+namespace moc_host {
+int eval_rows(const moc_graph* g, const int64_t* offs, const int32_t* seqs, const int32_t* lens, int32_t B,
+              int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st) {
+    if (!g->plan_eval.valid) {
+        int rc = make_plan(g, false, &g->plan_eval);
+        if (rc != MOC_OK) return rc;
+    }
+    const Plan& pl = g->plan_eval;
+    if (pl.global_state) {
+        int rc = ensure((void**)&g->d_state, &g->state_cap, (size_t)pl.grid * pl.group_bytes);
+        if (rc != MOC_OK) return rc;
+    }
+    return enqueue_eval(g, pl, const_cast<int64_t*>(offs), false, seqs, lens, B, M, out_peak, out_dur, out_feasible, st);
+}
+}  // namespace moc_host
 
 extern "C" {
 
@@ -741,7 +690,7 @@ int moc_eval_batch_noalloc(const moc_graph* g, const int32_t* seqs, const int32_
         return fail(MOC_ERR_ARG, "moc_eval_batch_noalloc: this graph needs a global workspace "
                     "(per-sequence state exceeds shared memory); use moc_eval_batch");
     // the offsets kernel rewrites offs[0..B] before the evaluation kernel reads them
-    return enqueue_eval(g, pl, offs, seqs, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream);
+    return enqueue_eval(g, pl, offs, true, seqs, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream);
 }
 
 int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t* out_profile,

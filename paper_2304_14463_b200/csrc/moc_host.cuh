@@ -1,0 +1,104 @@
+// Host-side types shared by the translation units of libmoc_b200.so: the graph handle, the launch
+// plan of the evaluation kernels, error reporting, and the one internal entry that enqueues an
+// evaluation with caller-supplied row offsets.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moc.h"
+#include "moc_kernels.cuh"
+#include "moc_pair_kernel.cuh"
+
+namespace moc_host {
+
+using KernelFn = void (*)(const moc::EvalParams);
+using PairFn = void (*)(const moc::PairParams);
+
+struct Plan {
+    bool valid = false;
+    KernelFn fn = nullptr;
+    int G = 0, gpc = 0, grid = 0, block = 0, CP = 0;
+    size_t smem = 0;
+    bool global_state = false, wide = false;
+    uint32_t cnt_bytes = 0, occ_bytes = 0, delta_bytes = 0, group_bytes = 0;
+    // fast path for C <= 2: a warp per sequence, graph staged in shared memory
+    bool pair = false;
+    PairFn pair_fn = nullptr;
+    uint32_t rec_bytes = 0, w_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
+};
+
+
+// Records the error text of the calling thread and returns `code`.
+int fail(int code, const char* fmt, ...);
+// Empties the error text of the calling thread (every entry point starts with this).
+void clear_error();
+// Counter behind moc_last_launch_count().
+int& launch_counter();
+
+#define MOC_CUDA(call)                                                                      \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return moc_host::fail(e_ == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, \
+                                  "%s: %s", #call, cudaGetErrorString(e_));                 \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace moc_host
+
+struct moc_graph {
+    int32_t n = 0;
+    int64_t n_edges = 0;  // distinct
+    int32_t C = 2;
+    int device = 0;
+    int sm_count = 0;
+    size_t smem_optin = 0;
+    int64_t sum_m = 0, sum_w = 0;
+    int32_t* d_succ_start = nullptr;
+    int32_t* d_succ = nullptr;
+    int64_t* d_w = nullptr;
+    int64_t* d_m64 = nullptr;
+    int32_t* d_m32 = nullptr;
+    int32_t want_G = 0, want_gpc = 0;
+    cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
+    // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
+    int32_t sell_len = 0, n_tiles = 0;
+    void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
+    void* d_rec64 = nullptr;
+    int64_t* d_wslot = nullptr;
+    uint32_t* d_sell = nullptr;
+    uint32_t* d_tile = nullptr;
+    // grow-only scratch; mutable because evaluation takes a const handle
+    mutable moc_host::Plan plan_eval, plan_profile;
+    mutable int64_t* d_offs = nullptr;
+    mutable size_t offs_cap = 0;
+    mutable char* d_state = nullptr;
+    mutable size_t state_cap = 0;
+    mutable int32_t* d_stage_seqs = nullptr;
+    mutable size_t stage_seqs_cap = 0;
+    mutable char* d_stage_io = nullptr;  // lens | peak | dur | status
+    mutable size_t stage_io_cap = 0;
+};
+
+
+namespace moc_host {
+
+// Enqueues the evaluation of B rows that start at seqs + offs[b] (offs: DEVICE, B+1 entries, the
+// last one the number of ints readable from seqs).  The handle's plan is made on first use and its
+// global workspace grown if the graph needs one.  Same outputs as moc_eval_batch.
+int eval_rows(const moc_graph* g, const int64_t* offs, const int32_t* seqs, const int32_t* lens, int32_t B,
+              int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st);
+
+}  // namespace moc_host

@@ -347,7 +347,7 @@ constexpr int kOffsThreads = 256;
 constexpr int kOffsPer = 4;
 constexpr int kOffsTile = kOffsThreads * kOffsPer;
 
-__global__ void __launch_bounds__(kOffsThreads) offsets_kernel(const int32_t* __restrict__ lens, int32_t B,
+static __global__ void __launch_bounds__(kOffsThreads) offsets_kernel(const int32_t* __restrict__ lens, int32_t B,
                                                                 int64_t* __restrict__ offs) {
     __shared__ int64_t wsum[kOffsThreads / 32];
     __shared__ int64_t wtot[kOffsThreads / 32];

@@ -1,0 +1,194 @@
+// Host side of the search entry points of libmoc_b200.so (declared in include/moc.h): state of the
+// chains on the device and the per-generation launch sequence.  Proposals, scoring and selection
+// all run in kernels (moc_search_kernels.cuh and the evaluation kernels).
+#include <algorithm>
+#include <new>
+
+#include "moc_host.cuh"
+#include "moc_search_kernels.cuh"
+
+using namespace moc_host;
+
+struct moc_search {
+    const moc_graph* g = nullptr;
+    int device = 0;
+    int32_t P = 0, stride = 0;
+    int64_t M = 0;
+    uint64_t seed = 0;
+    uint32_t generation = 0;   // generations completed (proposed, scored and settled)
+    char* d_block = nullptr;   // one allocation, carved up below
+    int32_t* d_bad = nullptr;
+    moc::SearchParams p{};
+};
+
+namespace {
+
+size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
+
+int chain_blocks(int32_t P) { return (P + moc::kSearchThreads / 32 - 1) / (moc::kSearchThreads / 32); }
+
+}  // namespace
+
+extern "C" {
+
+int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t P, int64_t M,
+                      uint64_t seed, void* stream, moc_search** out) {
+    clear_error();
+    launch_counter() = 0;
+    if (out) *out = nullptr;
+    if (!g || !out || !seqs || !lens || P < 1) return fail(MOC_ERR_ARG, "moc_search_create: null pointer or P < 1");
+    if (reinterpret_cast<uintptr_t>(seqs) & 3) return fail(MOC_ERR_ARG, "moc_search_create: seqs not 4-byte aligned");
+    const int64_t max_T = (int64_t)g->C * g->n;
+    const int64_t stride = (max_T + 3) & ~int64_t(3);
+    if (2 * (int64_t)P * stride > ((int64_t)1 << 40)) return fail(MOC_ERR_ARG, "moc_search_create: population too large");
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    moc_search* s = new (std::nothrow) moc_search();
+    if (!s) return fail(MOC_ERR_NOMEM, "host allocation failed");
+    s->g = g;
+    s->device = g->device;
+    s->P = P;
+    s->stride = (int32_t)stride;
+    s->M = M;
+    s->seed = seed;
+    const size_t bP = (size_t)P;
+    const size_t o_rows = 0, o_offs = o_rows + up256(2 * bP * (size_t)stride * 4), o_peak = o_offs + up256((bP + 1) * 8),
+                 o_dur = o_peak + up256(bP * 8), o_cpeak = o_dur + up256(bP * 8), o_cdur = o_cpeak + up256(bP * 8),
+                 o_cur = o_cdur + up256(bP * 8), o_lens = o_cur + up256(bP * 4), o_st = o_lens + up256(bP * 4),
+                 o_acc = o_st + up256(bP * 4), o_clens = o_acc + up256(bP * 4), o_cst = o_clens + up256(bP * 4),
+                 o_bad = o_cst + up256(bP * 4), total = o_bad + 256;
+    cudaError_t e = cudaMalloc((void**)&s->d_block, total);
+    if (e != cudaSuccess) {
+        delete s;
+        cudaGetLastError();
+        return fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, "moc_search_create: %s", cudaGetErrorString(e));
+    }
+    char* b = s->d_block;
+    moc::SearchParams& p = s->p;
+    p.P = P;
+    p.stride = (int32_t)stride;
+    p.max_T = (int32_t)max_T;
+    p.M = M;
+    p.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu);
+    p.seed_hi = (uint32_t)(seed >> 32);
+    p.generation = 0;
+    p.rows = (int32_t*)(b + o_rows);
+    p.c_offs = (int64_t*)(b + o_offs);
+    p.peak = (int64_t*)(b + o_peak);
+    p.dur = (int64_t*)(b + o_dur);
+    p.c_peak = (int64_t*)(b + o_cpeak);
+    p.c_dur = (int64_t*)(b + o_cdur);
+    p.cur = (int32_t*)(b + o_cur);
+    p.lens = (int32_t*)(b + o_lens);
+    p.status = (int32_t*)(b + o_st);
+    p.n_acc = (int32_t*)(b + o_acc);
+    p.c_lens = (int32_t*)(b + o_clens);
+    p.c_status = (int32_t*)(b + o_cst);
+    s->d_bad = (int32_t*)(b + o_bad);
+    int rc = MOC_OK;
+    int32_t bad = 0;
+    auto run = [&]() -> int {
+        MOC_CUDA(cudaMemsetAsync(s->d_bad, 0, 4, st));
+        // packed offsets of the caller's sequences, then the rows, then their evaluation
+        moc::offsets_kernel<<<(P + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, P, p.c_offs);
+        moc::search_init_kernel<<<chain_blocks(P), moc::kSearchThreads, 0, st>>>(p, seqs, lens, p.c_offs, s->d_bad);
+        moc::search_offsets_kernel<<<(P + 255) / 256, 256, 0, st>>>(p);
+        MOC_CUDA(cudaGetLastError());
+        int r = eval_rows(g, p.c_offs, p.rows, p.lens, P, M, p.peak, p.dur, p.status, st);
+        if (r != MOC_OK) return r;
+        MOC_CUDA(cudaMemcpyAsync(&bad, s->d_bad, 4, cudaMemcpyDeviceToHost, st));
+        MOC_CUDA(cudaStreamSynchronize(st));
+        return MOC_OK;
+    };
+    rc = run();
+    if (rc == MOC_OK && bad)
+        rc = fail(MOC_ERR_ARG, "moc_search_create: a sequence length lies outside [0, C*n = %lld]", (long long)max_T);
+    if (rc != MOC_OK) {
+        cudaFree(s->d_block);
+        delete s;
+        return rc;
+    }
+    *out = s;
+    return MOC_OK;
+}
+
+int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
+    clear_error();
+    launch_counter() = 0;
+    if (!s || n_generations < 0) return fail(MOC_ERR_ARG, "moc_search_run: null handle or negative count");
+    if ((uint64_t)s->generation + (uint64_t)n_generations > 0xFFFFFFFFull)
+        return fail(MOC_ERR_ARG, "moc_search_run: generation counter would pass 2^32 - 1");
+    if (n_generations == 0) return MOC_OK;
+    DeviceGuard dg(s->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    moc::SearchParams& p = s->p;
+    const int blocks = chain_blocks(s->P);
+    int launches = 0;
+    for (int32_t k = 0; k < n_generations; ++k) {
+        p.generation = s->generation + (uint32_t)k;
+        // settle the previous generation's proposals (none before the first one), propose the next
+        if (k == 0) moc::search_step_kernel<false, true><<<blocks, moc::kSearchThreads, 0, st>>>(p);
+        else moc::search_step_kernel<true, true><<<blocks, moc::kSearchThreads, 0, st>>>(p);
+        ++launches;
+        int rc = eval_rows(s->g, p.c_offs, p.rows, p.c_lens, s->P, s->M, p.c_peak, p.c_dur, p.c_status, st);
+        launches += launch_counter();
+        launch_counter() = 0;
+        if (rc != MOC_OK) return rc;
+    }
+    moc::search_step_kernel<true, false><<<blocks, moc::kSearchThreads, 0, st>>>(p);
+    ++launches;
+    MOC_CUDA(cudaGetLastError());
+    s->generation += (uint32_t)n_generations;
+    launch_counter() = launches;
+    return MOC_OK;
+}
+
+int moc_search_state(const moc_search* s, int32_t* out_rows, int32_t* out_lens, int64_t* out_peak,
+                     int64_t* out_dur, int32_t* out_status, int32_t* out_accepted, void* stream) {
+    clear_error();
+    if (!s) return fail(MOC_ERR_ARG, "moc_search_state: null handle");
+    DeviceGuard dg(s->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", s->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bP = (size_t)s->P;
+    if (out_rows) {
+        moc::search_export_kernel<<<chain_blocks(s->P), moc::kSearchThreads, 0, st>>>(s->p, out_rows);
+        MOC_CUDA(cudaGetLastError());
+    }
+    if (out_lens) MOC_CUDA(cudaMemcpyAsync(out_lens, s->p.lens, bP * 4, cudaMemcpyDeviceToDevice, st));
+    if (out_peak) MOC_CUDA(cudaMemcpyAsync(out_peak, s->p.peak, bP * 8, cudaMemcpyDeviceToDevice, st));
+    if (out_dur) MOC_CUDA(cudaMemcpyAsync(out_dur, s->p.dur, bP * 8, cudaMemcpyDeviceToDevice, st));
+    if (out_status) MOC_CUDA(cudaMemcpyAsync(out_status, s->p.status, bP * 4, cudaMemcpyDeviceToDevice, st));
+    if (out_accepted) MOC_CUDA(cudaMemcpyAsync(out_accepted, s->p.n_acc, bP * 4, cudaMemcpyDeviceToDevice, st));
+    return MOC_OK;
+}
+
+int moc_search_best(const moc_search* s, int32_t* out_seq, int64_t* out_best, void* stream) {
+    clear_error();
+    if (!s || !out_best) return fail(MOC_ERR_ARG, "moc_search_best: null handle or null out_best");
+    DeviceGuard dg(s->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", s->device);
+    moc::search_best_kernel<<<1, moc::kBestThreads, 0, (cudaStream_t)stream>>>(s->p, out_seq, out_best);
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+
+int moc_search_info(const moc_search* s, int32_t* P, int32_t* stride, uint32_t* generation) {
+    clear_error();
+    if (!s) return fail(MOC_ERR_ARG, "moc_search_info: null handle");
+    if (P) *P = s->P;
+    if (stride) *stride = s->stride;
+    if (generation) *generation = s->generation;
+    return MOC_OK;
+}
+
+void moc_search_destroy(moc_search* s) {
+    if (!s) return;
+    DeviceGuard dg(s->device);
+    cudaFree(s->d_block);
+    delete s;
+}
+
+}  // extern "C"

@@ -1,0 +1,120 @@
+"""Parity of the search entry points (through the C ABI) with the search oracle: after any number of
+generations every chain's sequence, length, evaluation and acceptance count are identical."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import OracleGraph, OracleSearch
+from paper_2304_14463_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2304_14463_b200 import build
+    build.build()
+    from paper_2304_14463_b200 import binding
+    return binding
+
+
+def dev(a, dtype=torch.int32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype).cuda()
+
+
+def assert_state_equal(S, OS, what=""):
+    st = S.state()
+    torch.cuda.synchronize()
+    lens = st["lens"].cpu().numpy()
+    assert (lens == OS.lens).all(), f"{what}: lengths differ at {np.nonzero(lens != OS.lens)[0][:5]}"
+    for k, want in (("peak", OS.peak), ("dur", OS.dur), ("status", OS.status)):
+        got = st[k].cpu().numpy()
+        assert (got == want).all(), f"{what}: {k} differs at {np.nonzero(got != want)[0][:5]}"
+    rows = st["rows"].cpu().numpy()
+    for c in range(OS.P):
+        assert (rows[c, :lens[c]] == OS.pop[c, :lens[c]]).all(), f"{what}: sequence of chain {c} differs"
+    assert int(st["accepted"].sum()) == OS.accepted
+    b = S.best()
+    ob = OS.best()
+    assert b["index"] == ob and b["accepted"] == OS.accepted
+    if ob >= 0:
+        assert (b["peak"], b["dur"], b["status"]) == (int(OS.peak[ob]), int(OS.dur[ob]), int(OS.status[ob]))
+        assert (b["seq"] == OS.row(ob)).all()
+
+
+def make_pair(B, wl, seqs, lens, M, seed):
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    S = B.Search(G, dev(seqs), dev(lens), M, seed)
+    OS = OracleSearch(O, seqs, lens, M, seed, stride=S.info()["stride"])
+    return G, O, S, OS
+
+
+@pytest.mark.parametrize("idx,P,gens", [(0, 1024, (1, 2, 40)), (1, 512, (1, 9, 20)), (2, 384, (1, 6, 25)),
+                                        (3, 96, (1, 5)), (4, 24, (1, 4))])
+def test_search_parity(B, idx, P, gens):
+    """Every configuration (C = 2 warp kernel and C = 3 group kernel), 1/16 of the start population
+    damaged, budget 80 % of the no-rematerialization peak; state compared after each call."""
+    wl = W.make(idx, seed=1, B=P)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=5, frac=1 / 16)
+    assert (lens <= wl.C * wl.n).all()
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G, O, S, OS = make_pair(B, wl, seqs, lens, M, seed=(idx + 1) * 0x9E3779B97F4A7C15 % (1 << 64))
+    assert_state_equal(S, OS, "start")
+    for g in gens:
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"config {idx} after {OS.generation} generations")
+    assert S.info()["generation"] == OS.generation
+    assert OS.accepted > 0
+
+
+def test_search_from_identity_reaches_budget(B):
+    """Chains that all start from the identity order: over budget at first (Phase 1), then feasible
+    chains only trade duration (Phase 2); the key of every chain never increases."""
+    wl = W.make(0, seed=2, B=256)
+    n = wl.n
+    seqs = np.tile(np.arange(n, dtype=np.int32), 256)
+    lens = np.full(256, n, np.int32)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    P0 = O0.eval(np.arange(n), 1 << 60)["peak"]
+    M = P0 * 90 // 100
+    G, O, S, OS = make_pair(B, wl, seqs, lens, M, seed=77)
+    prev = None
+    for g in (10, 50, 200):
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"after {OS.generation}")
+        key = np.stack([np.maximum(OS.peak, M), OS.dur], 1)
+        if prev is not None:
+            assert ((key[:, 0] < prev[:, 0]) | ((key[:, 0] == prev[:, 0]) & (key[:, 1] <= prev[:, 1]))).all()
+        prev = key
+
+
+def test_search_split_invariance_and_errors(B):
+    wl = W.make(2, seed=3, B=64)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    a = B.Search(G, dev(wl.seqs), dev(wl.lens), M, 5)
+    b = B.Search(G, dev(wl.seqs), dev(wl.lens), M, 5)
+    a.run(12)
+    for k in (0, 5, 1, 6):
+        b.run(k)
+    sa, sb = a.state(), b.state()
+    torch.cuda.synchronize()
+    for k in ("rows", "lens", "peak", "dur", "status", "accepted"):
+        assert torch.equal(sa[k], sb[k])
+    assert B.moc_last_launch_count() >= 0
+    # a length beyond C*n is refused
+    lens = wl.lens.copy()
+    seqs = np.concatenate([wl.seqs, np.zeros(2 * wl.C * wl.n, np.int32)])
+    lens[-1] = wl.C * wl.n + 1
+    with pytest.raises(B.MocError) as e:
+        B.Search(G, dev(seqs), dev(lens), M, 5)
+    assert e.value.code == -1
+    # an all-invalid population has no best chain
+    bad = np.zeros(4 * wl.n, np.int32)
+    s = B.Search(G, dev(bad), dev(np.full(4, wl.n, np.int32)), M, 1)
+    assert s.best()["index"] == -1
