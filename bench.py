@@ -149,6 +149,87 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_search(args):
+    """Throughput of the search entry points: generations of P chains on the headline graph.  Prints a
+    JSON line of its own (the default run's line is the evaluation metric)."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --mode search needs a CUDA device")
+    torch.cuda.set_device(0)
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2304_14463_b200 import binding, workloads
+    P = args.chains
+    base = workloads.make(WORKLOAD_IDX, seed=1, B=P)
+    G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
+    P0 = G.no_remat_peak()
+    M = binding.budget_from_peak(P0, PCT)
+    d_seqs, d_lens = torch.from_numpy(base.seqs).cuda(), torch.from_numpy(base.lens).cuda()
+    S = binding.Search(G, d_seqs, d_lens, M, seed=1)
+    stride = S.info()["stride"]
+    steps, warm = (200 if args.steps is None else args.steps), max(3, 20 if args.warmup is None else args.warmup)
+    S.run(warm)
+    per_call = binding.moc_last_launch_count()
+    torch.cuda.synchronize()
+    lens0 = S.state(want_rows=False)["lens"].double().sum().item()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream = torch.cuda.current_stream()
+    with ClockSampler(0) as clocks:
+        e0.record(stream)
+        S.run(steps)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    launches = binding.moc_last_launch_count()
+    lens1 = S.state(want_rows=False)["lens"].double().sum().item()
+    mean_T = 0.5 * (lens0 + lens1) / P
+    best = S.best()
+    # bytes one generation has to move: proposal kernel reads the row and writes the proposal,
+    # the evaluation reads the proposal; per chain about 60 bytes of state and results
+    alg_bytes = P * (3 * 4 * mean_T + 100)
+    peak_gbs, peak_kind = load_peaks()
+    sum_w = int(base.w.sum())
+    line = {"metric": "search_proposals_per_s_n442", "value": P * steps / (ms * 1e-3), "unit": "proposals/s",
+            "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": f"search on {base.name}: n={base.n} m={len(base.edges)} C={base.C} chains={P} "
+                                   f"M={PCT}% of no-remat peak ({M})", "mean_T": mean_T,
+                       "cold_l2": f"rows of the chains: {2 * P * stride * 4 / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2"},
+            "schedule_steps_per_s": P * mean_T * steps / (ms * 1e-3),
+            "gpu_launches": launches, "launches_per_generation": (per_call - 1) / warm,
+            "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms / steps * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
+                         "frac": alg_bytes / (ms / steps * 1e-3) / 1e9 / peak_gbs, "peak_kind": f"of {peak_kind}",
+                         "traffic": None, "algorithmic_bytes_per_generation": alg_bytes,
+                         "note": "whole generation (proposal kernel + evaluation kernel), not one kernel"},
+            "result": {"generations": S.info()["generation"], "best_status": best["status"], "best_peak": best["peak"],
+                       "best_dur": best["dur"], "tdi_percent": 100.0 * (best["dur"] - sum_w) / sum_w if best["index"] >= 0 else None,
+                       "accepted": best["accepted"], "no_remat_peak": P0, "budget": M},
+            "clocks": clocks.summary()}
+    if not args.no_cpu_baseline:
+        from oracle import OracleGraph, OracleSearch
+        Pc = min(P, 1024)
+        O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
+        offs = np.concatenate([[0], np.cumsum(base.lens)])
+        OS = OracleSearch(O, base.seqs[:offs[Pc]], base.lens[:Pc], M, seed=1, stride=stride)
+        OS.run(1)
+        t0, gens = time.perf_counter(), 0
+        while time.perf_counter() - t0 < 8.0:
+            OS.run(4)
+            gens += 4
+        dt = time.perf_counter() - t0
+        # parity of the sample: the same chains, the same number of generations, on the GPU
+        S2 = binding.Search(G, torch.from_numpy(base.seqs[:offs[Pc]]).cuda(), d_lens[:Pc].contiguous(), M, seed=1)
+        S2.run(OS.generation)
+        st = S2.state()
+        torch.cuda.synchronize()
+        same = bool((st["lens"].cpu().numpy() == OS.lens).all() and (st["peak"].cpu().numpy() == OS.peak).all()
+                    and (st["dur"].cpu().numpy() == OS.dur).all() and (st["status"].cpu().numpy() == OS.status).all())
+        line["cpu_baseline"] = {"value": Pc * gens / dt, "unit": "proposals/s", "cores": 1, "kind": "oracle",
+                                "sample": f"{Pc} chains, {gens} generations, one core (the search oracle is sequential)"}
+        line["parity_sample"] = same
+    print(json.dumps(line))
+
+
 def time_oracle(base, M, budget_s=6.0):
     from oracle import OracleGraph
     O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
@@ -179,7 +260,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", type=int, default=WORKLOAD_IDX,
                     help="index 0..4 of the configuration to time (default: the headline one)")
+    ap.add_argument("--mode", default="eval", choices=["eval", "search"],
+                    help="eval: the headline evaluation metric; search: generations of the search entry points")
+    ap.add_argument("--chains", type=int, default=32768, help="--mode search: number of chains")
     args = ap.parse_args()
+    if args.mode == "search" and args.impl != "reference":
+        return run_search(args)
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
