@@ -18,7 +18,8 @@
  *
  * Random draws: one call of Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers:
  * as easy as 1, 2, 3", SC 2011) per chain and generation, counter = (generation, chain, 0, 0),
- * key = (low, high) 32 bits of the seed.  The four output words r0..r3 select the edit:
+ * key = (low, high) 32 bits of the seed; "chain" is the chain's global number chain0 + c, so that a
+ * population split over several runs (one per device) draws what the unsplit population draws.  The four output words r0..r3 select the edit:
  *     op = r0 mod 3                 0 insert, 1 delete, 2 move
  *     q  = r1 mod T                 position of the copy the edit refers to
  *     insert:  j = r2 mod (T+1);  the node seq[q] is inserted in front of index j     (T+1 steps)
@@ -111,11 +112,12 @@ int32_t moc_oracle_accept(int64_t peak_c, int64_t dur_c, int32_t st_c, int64_t p
  *           is refused before it is stored)
  *   lens    P lengths;  peak, dur, status: the evaluation of every chain's current sequence
  *           (the caller evaluates the initial population).
+ *   chain0  global number of chain 0 (enters the random draws only).
  *   n_accepted (may be NULL) receives the number of accepted proposals.
  */
 void moc_oracle_search_run(const void *g, int32_t *pop, int32_t *lens, int64_t *peak, int64_t *dur,
                            int32_t *status, int32_t P, int32_t stride, int64_t M, uint64_t seed,
-                           uint32_t gen0, uint32_t n_gen, int64_t *n_accepted) {
+                           uint32_t gen0, uint32_t n_gen, uint32_t chain0, int64_t *n_accepted) {
     int32_t *child = (int32_t *)malloc(((size_t)stride + 2) * sizeof(int32_t));
     const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
     int64_t acc = 0;
@@ -123,7 +125,7 @@ void moc_oracle_search_run(const void *g, int32_t *pop, int32_t *lens, int64_t *
         for (int32_t c = 0; c < P; ++c) {
             int32_t *row = pop + (size_t)c * stride;
             const int32_t T = lens[c];
-            const uint32_t ctr[4] = {gen, (uint32_t)c, 0u, 0u};
+            const uint32_t ctr[4] = {gen, chain0 + (uint32_t)c, 0u, 0u};
             uint32_t r[4];
             moc_oracle_philox4x32_10(ctr, key, r);
             const int32_t Tc = moc_oracle_mutate(row, T, r[0], r[1], r[2], child);

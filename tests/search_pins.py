@@ -102,7 +102,7 @@ def _tiny_problem():
     return n, edges, w, m
 
 
-def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen):
+def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen, chain0=0):
     """The generation loop restated in Python over the separately pinned pieces, with the
     set-definition evaluator of defs.py in place of the oracle's evaluator."""
     def ev(s):
@@ -113,7 +113,7 @@ def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, ge
     key = [seed & 0xFFFFFFFF, seed >> 32]
     for gen in range(gen0, gen0 + n_gen):
         for c, r in enumerate(rows):
-            x = oracle.philox4x32_10([gen, c, 0, 0], key, lib=lib)
+            x = oracle.philox4x32_10([gen, chain0 + c, 0, 0], key, lib=lib)
             child = list_edit(r, int(x[0]), int(x[1]), int(x[2]))
             if child is None:
                 continue
@@ -134,12 +134,13 @@ def pin_search_loop(make_graph, lib):
             rows = [list(range(n)) for _ in range(6)] + [[0, 1, 2, 0, 3, 4], [4, 3, 2, 1, 0], [0, 1, 2]]
             seqs = np.array([x for r in rows for x in r], np.int32)
             lens = np.array([len(r) for r in rows], np.int32)
-            S = oracle.OracleSearch(g, seqs, lens, M, seed)
+            chain0 = 0 if M == P0 else 1000
+            S = oracle.OracleSearch(g, seqs, lens, M, seed, chain0=chain0)
             done = 0
             for n_gen in (1, 7, 40):
                 before = [key_of((S.peak[c], S.dur[c], S.status[c]), M) for c in range(S.P)]
                 S.run(n_gen)
-                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen)
+                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen, chain0)
                 done += n_gen
                 for c in range(S.P):
                     assert list(S.row(c)) == want_rows[c], (M, seed, c)
@@ -186,6 +187,15 @@ def pin_search_reaches_optimum(make_graph, lib):
     S2.run(300)
     for c in (0, 2, 31):
         assert list(S2.row(c)) == list(S.row(c))
+    # a population split in two (second half numbered from chain0 = 16) gives the same chains
+    half = P // 2
+    Sa = oracle.OracleSearch(g, seqs[:half * n], lens[:half], M, seed=11)
+    Sb = oracle.OracleSearch(g, seqs[half * n:], lens[half:], M, seed=11, chain0=half)
+    Sa.run(300)
+    Sb.run(300)
+    for c in range(P):
+        part, k = (Sa, c) if c < half else (Sb, c - half)
+        assert list(part.row(k)) == list(S.row(c))
 
 
 def run_all(make_graph, lib):
