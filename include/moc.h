@@ -174,8 +174,8 @@ int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t
  * chain can drift across plateaus.
  *
  * Proposal of chain c in generation k for a sequence of T steps (T = 0 proposes nothing): with
- * (r0, r1, r2, r3) = Philox4x32-10(counter = (k, c, 0, 0), key = (seed mod 2^32, seed div 2^32))
- * (Salmon, Moraes, Dror, Shaw, SC 2011),
+ * (r0, r1, r2, r3) = Philox4x32-10(counter = (k, first_chain + c, 0, 0), key = (seed mod 2^32,
+ * seed div 2^32)) (Salmon, Moraes, Dror, Shaw, SC 2011),
  *     op = r0 mod 3, q = r1 mod T;
  *     op 0  insert: a further copy of node seq[q] is put in front of index j = r2 mod (T+1);
  *     op 1  delete: element q is removed;
@@ -197,11 +197,15 @@ typedef struct moc_search moc_search; /* opaque */
  *                (MOC_ERR_ARG otherwise).  Sequences may be invalid (status < 0): such a chain
  *                accepts the first proposal with status >= 0.
  *   M            memory budget;  seed: key of the random draws.
+ *   first_chain  global number of chain 0.  A population split over several handles (one per
+ *                GPU) evolves exactly like the unsplit one when every part is given the global
+ *                number of its first chain; 0 for a single handle.  first_chain + P <= 2^32.
  * Copies the sequences, evaluates them and synchronises `stream` before returning.
  * Errors: MOC_ERR_ARG, MOC_ERR_CUDA, MOC_ERR_NOMEM; *out is NULL on error.
  */
 int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t P,
-                      int64_t M, uint64_t seed, void* stream, moc_search** out);
+                      int64_t M, uint64_t seed, uint32_t first_chain, void* stream,
+                      moc_search** out);
 
 /* Enqueues n_generations further generations on `stream` (asynchronous; two kernels per generation
  * plus one at the end, no allocation, no synchronisation).  Generations are numbered from 0 over

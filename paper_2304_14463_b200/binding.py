@@ -49,7 +49,7 @@ lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
 lib.moc_graph_set_timing_events.restype = ctypes.c_int
 lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
 lib.moc_search_create.restype = ctypes.c_int
-lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, _P, ctypes.POINTER(_P)]
+lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, ctypes.c_uint32, _P, ctypes.POINTER(_P)]
 lib.moc_search_run.restype = ctypes.c_int
 lib.moc_search_run.argtypes = [_P, _i32, _P]
 lib.moc_search_state.restype = ctypes.c_int
@@ -223,12 +223,13 @@ def moc_last_launch_count():
     return lib.moc_last_launch_count()
 
 
-def moc_search_create(g, seqs, lens, M, seed):
+def moc_search_create(g, seqs, lens, M, seed, first_chain=0):
     """Device tensors (packed sequences, lengths) -> search handle; synchronous."""
     import torch
     h = _P()
     rc = lib.moc_search_create(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"), lens.numel(),
-                               int(M), ctypes.c_uint64(int(seed)), _stream(), ctypes.byref(h))
+                               int(M), ctypes.c_uint64(int(seed)), ctypes.c_uint32(int(first_chain)), _stream(),
+                               ctypes.byref(h))
     _check(rc, "moc_search_create")
     return h
 
@@ -331,10 +332,10 @@ class Graph:
 class Search:
     """Owns a moc_search handle; keeps its Graph alive."""
 
-    def __init__(self, graph: Graph, seqs, lens, M, seed):
+    def __init__(self, graph: Graph, seqs, lens, M, seed, first_chain=0):
         self.graph = graph
         self.M = int(M)
-        self.h = moc_search_create(graph.h, seqs, lens, M, seed)
+        self.h = moc_search_create(graph.h, seqs, lens, M, seed, first_chain)
 
     def close(self, _destroy=lib.moc_search_destroy):
         if getattr(self, "h", None):

@@ -32,7 +32,7 @@ int chain_blocks(int32_t P) { return (P + moc::kSearchThreads / 32 - 1) / (moc::
 extern "C" {
 
 int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t P, int64_t M,
-                      uint64_t seed, void* stream, moc_search** out) {
+                      uint64_t seed, uint32_t first_chain, void* stream, moc_search** out) {
     clear_error();
     launch_counter() = 0;
     if (out) *out = nullptr;
@@ -40,6 +40,8 @@ int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* le
     if (reinterpret_cast<uintptr_t>(seqs) & 3) return fail(MOC_ERR_ARG, "moc_search_create: seqs not 4-byte aligned");
     const int64_t max_T = (int64_t)g->C * g->n;
     const int64_t stride = (max_T + 3) & ~int64_t(3);
+    if ((uint64_t)first_chain + (uint64_t)P > 0x100000000ull)
+        return fail(MOC_ERR_ARG, "moc_search_create: first_chain + P exceeds 2^32");
     if (2 * (int64_t)P * stride > ((int64_t)1 << 40)) return fail(MOC_ERR_ARG, "moc_search_create: population too large");
     DeviceGuard dg(g->device);
     if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
@@ -73,6 +75,7 @@ int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* le
     p.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu);
     p.seed_hi = (uint32_t)(seed >> 32);
     p.generation = 0;
+    p.chain0 = first_chain;
     p.rows = (int32_t*)(b + o_rows);
     p.c_offs = (int64_t*)(b + o_offs);
     p.peak = (int64_t*)(b + o_peak);

@@ -14,7 +14,8 @@
 // array of row offsets that the proposing kernel writes.
 //
 // Random draws: one block of Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC 2011) per chain and
-// generation with counter (generation, chain, 0, 0) and the 64-bit seed as the key.
+// generation with counter (generation, chain0 + chain, 0, 0) and the 64-bit seed as the key; chain0
+// numbers the chains globally when a population is split over several devices.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -44,6 +45,7 @@ struct SearchParams {
     int64_t M;
     uint32_t seed_lo, seed_hi;
     uint32_t generation; // of the proposals written by this launch
+    uint32_t chain0;     // global number of chain 0 (enters the random draws only)
     int32_t* rows;       // 2 * P * stride
     int32_t* cur;        // P: 0 or 1
     int32_t* lens;       // P: length of each chain's sequence
@@ -112,7 +114,7 @@ __global__ void __launch_bounds__(kSearchThreads) search_step_kernel(const Searc
         if (lane == 0) p.c_lens[c] = 0;
         return;
     }
-    const uint4 r = philox4x32_10(make_uint4(p.generation, (uint32_t)c, 0u, 0u), make_uint2(p.seed_lo, p.seed_hi));
+    const uint4 r = philox4x32_10(make_uint4(p.generation, p.chain0 + (uint32_t)c, 0u, 0u), make_uint2(p.seed_lo, p.seed_hi));
     const uint32_t op = r.x % 3u;
     const int32_t q = (int32_t)(r.y % (uint32_t)T);
     // The proposal is "take element q out (delete, move), then put x in front of index j (insert,

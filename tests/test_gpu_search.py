@@ -107,6 +107,17 @@ def test_search_split_invariance_and_errors(B):
     for k in ("rows", "lens", "peak", "dur", "status", "accepted"):
         assert torch.equal(sa[k], sb[k])
     assert B.moc_last_launch_count() >= 0
+    # a population split over two handles evolves like the unsplit one
+    half = 32
+    offs = np.concatenate([[0], np.cumsum(wl.lens)])
+    lo = B.Search(G, dev(wl.seqs[:offs[half]]), dev(wl.lens[:half]), M, 5)
+    hi = B.Search(G, dev(wl.seqs[offs[half]:]), dev(wl.lens[half:]), M, 5, first_chain=half)
+    lo.run(12)
+    hi.run(12)
+    sl, sh = lo.state(), hi.state()
+    torch.cuda.synchronize()
+    for k in ("rows", "lens", "peak", "dur", "status", "accepted"):
+        assert torch.equal(torch.cat([sl[k], sh[k]]), sa[k])
     # a length beyond C*n is refused
     lens = wl.lens.copy()
     seqs = np.concatenate([wl.seqs, np.zeros(2 * wl.C * wl.n, np.int32)])

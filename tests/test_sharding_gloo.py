@@ -62,3 +62,57 @@ def test_shard_ranges():
             assert r[0][0] == 0 and r[-1][1] == B and all(a[1] == b[0] for a, b in zip(r, r[1:]))
             assert max(b - a for a, b in r) - min(b - a for a, b in r) <= 1
     assert sharding.aggregate_throughput([10, 30], [1.0, 2.0]) == 20.0
+
+
+def _search_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from oracle import OracleGraph, OracleSearch
+    from paper_2304_14463_b200 import sharding, workloads
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = workloads.make(0, seed=4, B=97, n_threads=1)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O.eval(np.arange(wl.n), 1 << 60)["peak"] * 85 // 100
+    out = []
+    for case in ("normal", "rank0_all_invalid"):
+        seqs, lens = wl.seqs.copy(), wl.lens.copy()
+        if case == "rank0_all_invalid":
+            b0, b1 = sharding.shard_range(len(lens), 0, world)
+            offs = np.concatenate([[0], np.cumsum(lens)])
+            seqs[:offs[b1]] = 0                             # rank 0 starts with invalid chains only
+        my_seqs, my_lens = sharding.shard_batch(seqs, lens, rank, world)
+        b0, _ = sharding.shard_range(len(lens), rank, world)
+        S = OracleSearch(O, my_seqs, my_lens, M, seed=9, chain0=b0)   # the oracle stands in for the device
+        S.run(0 if case == "rank0_all_invalid" else 60)
+        b = S.best()
+        mine = dict(index=b, peak=int(S.peak[b]) if b >= 0 else -1, dur=int(S.dur[b]) if b >= 0 else -1,
+                    status=int(S.status[b]) if b >= 0 else -2, seq=S.row(b) if b >= 0 else np.zeros(0, np.int32))
+        got = sharding.best_over_ranks(mine, M, b0, wl.C * wl.n)
+        if rank == 0:
+            full = OracleSearch(O, seqs, lens, M, seed=9)
+            full.run(0 if case == "rank0_all_invalid" else 60)
+            fb = full.best()
+            out.append(got["index"] == fb and (got["seq"] == full.row(fb)).all()
+                       and (got["peak"], got["dur"], got["status"]) == (int(full.peak[fb]), int(full.dur[fb]), int(full.status[fb]))
+                       and (case == "normal" or got["rank"] == 1))
+    if rank == 0:
+        q.put(out)
+    dist.destroy_process_group()
+
+
+def test_two_ranks_search_best():
+    """A population split over two ranks (global chain numbers) evolves like the unsplit one, and the
+    best chain over the ranks is the unsplit best, also when one rank has no valid chain."""
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_search_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    out = q.get(timeout=180)
+    for p in procs:
+        p.join(60)
+        assert p.exitcode == 0
+    assert out == [True, True]
