@@ -50,11 +50,11 @@ def load_library(path):
         lib.moc_oracle_philox4x32_10.restype = None
         lib.moc_oracle_philox4x32_10.argtypes = [P, P, P]
         lib.moc_oracle_mutate.restype = i32
-        lib.moc_oracle_mutate.argtypes = [P, i32, u32, u32, u32, P]
+        lib.moc_oracle_mutate.argtypes = [P, i32, u32, u32, u32, u32, P]
         lib.moc_oracle_accept.restype = i32
         lib.moc_oracle_accept.argtypes = [i64, i64, i32, i64, i64, i32, i64]
         lib.moc_oracle_search_run.restype = None
-        lib.moc_oracle_search_run.argtypes = [P, P, P, P, P, P, i32, i32, i64, u64, u32, u32, u32, P]
+        lib.moc_oracle_search_run.argtypes = [P, P, P, P, P, P, i32, i32, i64, u64, u32, u32, u32, u32, P]
         lib.moc_oracle_search_best.restype = i32
         lib.moc_oracle_search_best.argtypes = [P, P, P, i32, i64]
     return lib
@@ -132,12 +132,13 @@ def philox4x32_10(ctr, key, lib=None):
     return out
 
 
-def mutate(seq, r0, r1, r2, lib=None):
-    """The proposal the draws (r0, r1, r2) make from ``seq``; None for an empty sequence."""
+def mutate(seq, r0, r1, r2, kinds=7, lib=None):
+    """The proposal the draws (r0, r1, r2) make from ``seq`` with the enabled kinds of edit (bit 0
+    insert, bit 1 delete, bit 2 move); None for an empty sequence."""
     lib = lib if lib is not None else _load()
     seq = np.ascontiguousarray(seq, dtype=np.int32)
     child = np.zeros(len(seq) + 2, np.int32)
-    Tc = lib.moc_oracle_mutate(_ptr(seq), len(seq), int(r0), int(r1), int(r2), _ptr(child))
+    Tc = lib.moc_oracle_mutate(_ptr(seq), len(seq), int(r0), int(r1), int(r2), int(kinds), _ptr(child))
     return None if Tc < 0 else child[:Tc].copy()
 
 
@@ -151,12 +152,13 @@ def accept(child, parent, M, lib=None):
 class OracleSearch:
     """P chains of the search: rows of ``stride`` ints with lengths and evaluations."""
 
-    def __init__(self, graph: OracleGraph, seqs, lens, M, seed, stride=None, chain0=0):
+    def __init__(self, graph: OracleGraph, seqs, lens, M, seed, stride=None, chain0=0, kinds=7):
         self.g = graph
         self._lib = graph._lib
         self.M = int(M)
         self.seed = int(seed)
         self.chain0 = int(chain0)
+        self.kinds = int(kinds)
         lens = np.ascontiguousarray(lens, dtype=np.int32)
         self.P = len(lens)
         self.stride = int(stride) if stride is not None else graph.C * graph.n
@@ -174,7 +176,7 @@ class OracleSearch:
         acc = np.zeros(1, np.int64)
         self._lib.moc_oracle_search_run(self.g._h, _ptr(self.pop), _ptr(self.lens), _ptr(self.peak),
                                         _ptr(self.dur), _ptr(self.status), self.P, self.stride, self.M,
-                                        self.seed, self.generation, int(n_gen), self.chain0, _ptr(acc))
+                                        self.seed, self.generation, int(n_gen), self.chain0, self.kinds, _ptr(acc))
         self.generation += int(n_gen)
         self.accepted += int(acc[0])
         return int(acc[0])

@@ -20,7 +20,10 @@
  * as easy as 1, 2, 3", SC 2011) per chain and generation, counter = (generation, chain, 0, 0),
  * key = (low, high) 32 bits of the seed; "chain" is the chain's global number chain0 + c, so that a
  * population split over several runs (one per device) draws what the unsplit population draws.  The four output words r0..r3 select the edit:
- *     op = r0 mod 3                 0 insert, 1 delete, 2 move
+ *     op = r0 mod 3                 0 insert, 1 delete, 2 move   (with all three kinds enabled; with
+ *                                   a mask of k enabled kinds: the (r0 mod k)-th enabled one in
+ *                                   this order.  "move" alone searches over the orders of a
+ *                                   sequence without adding or removing copies.)
  *     q  = r1 mod T                 position of the copy the edit refers to
  *     insert:  j = r2 mod (T+1);  the node seq[q] is inserted in front of index j     (T+1 steps)
  *     delete:  element q is removed                                                   (T-1 steps)
@@ -68,13 +71,19 @@ void moc_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint
 }
 
 /*
- * Applies the edit selected by (r0, r1, r2) to seq[0..T) and writes the proposal to child (room
- * for T+1 ints).  Returns the proposal's length, or -1 when T = 0 (nothing to edit).
+ * Applies the edit selected by (r0, r1, r2) among the enabled kinds to seq[0..T) and writes the
+ * proposal to child (room for T+1 ints).  Returns the proposal's length, or -1 when T = 0 or no
+ * kind is enabled (nothing to edit).
  */
 int32_t moc_oracle_mutate(const int32_t *seq, int32_t T, uint32_t r0, uint32_t r1, uint32_t r2,
-                          int32_t *child) {
+                          uint32_t kinds, int32_t *child) {
     if (T <= 0) return -1;
-    const uint32_t op = r0 % 3u;
+    /* kinds: bit 0 insert, bit 1 delete, bit 2 move; at least one is set */
+    uint32_t enabled[3], k = 0;
+    for (uint32_t o = 0; o < 3; ++o)
+        if (kinds & (1u << o)) enabled[k++] = o;
+    if (k == 0) return -1;
+    const uint32_t op = enabled[r0 % k];
     const int32_t q = (int32_t)(r1 % (uint32_t)T);
     if (op == 0) { /* insert a further copy of seq[q] in front of index j */
         const int32_t j = (int32_t)(r2 % ((uint32_t)T + 1u));
@@ -113,11 +122,13 @@ int32_t moc_oracle_accept(int64_t peak_c, int64_t dur_c, int32_t st_c, int64_t p
  *   lens    P lengths;  peak, dur, status: the evaluation of every chain's current sequence
  *           (the caller evaluates the initial population).
  *   chain0  global number of chain 0 (enters the random draws only).
+ *   kinds   enabled kinds of edit (bit 0 insert, bit 1 delete, bit 2 move).
  *   n_accepted (may be NULL) receives the number of accepted proposals.
  */
 void moc_oracle_search_run(const void *g, int32_t *pop, int32_t *lens, int64_t *peak, int64_t *dur,
                            int32_t *status, int32_t P, int32_t stride, int64_t M, uint64_t seed,
-                           uint32_t gen0, uint32_t n_gen, uint32_t chain0, int64_t *n_accepted) {
+                           uint32_t gen0, uint32_t n_gen, uint32_t chain0, uint32_t kinds,
+                           int64_t *n_accepted) {
     int32_t *child = (int32_t *)malloc(((size_t)stride + 2) * sizeof(int32_t));
     const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
     int64_t acc = 0;
@@ -128,7 +139,7 @@ void moc_oracle_search_run(const void *g, int32_t *pop, int32_t *lens, int64_t *
             const uint32_t ctr[4] = {gen, chain0 + (uint32_t)c, 0u, 0u};
             uint32_t r[4];
             moc_oracle_philox4x32_10(ctr, key, r);
-            const int32_t Tc = moc_oracle_mutate(row, T, r[0], r[1], r[2], child);
+            const int32_t Tc = moc_oracle_mutate(row, T, r[0], r[1], r[2], kinds, child);
             if (Tc < 0) continue;
             int64_t pk, du;
             int32_t st;

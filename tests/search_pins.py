@@ -24,13 +24,14 @@ def pin_philox_kat(lib):
         assert [int(x) for x in out] == v[6:10], (r, [hex(int(x)) for x in out])
 
 
-def list_edit(seq, r0, r1, r2):
+def list_edit(seq, r0, r1, r2, kinds=7):
     """The three edits restated with Python list operations."""
     s = list(seq)
     T = len(s)
     if T == 0:
         return None
-    op, q = r0 % 3, r1 % T
+    enabled = [o for o in range(3) if kinds >> o & 1]
+    op, q = enabled[r0 % len(enabled)], r1 % T
     if op == 0:
         s.insert(r2 % (T + 1), s[q])
     elif op == 1:
@@ -73,6 +74,15 @@ def pin_edits(lib):
         # the multiset changes by exactly the edit's element
         op = r[0] % 3
         assert len(got) == T + (1, -1, 0)[op]
+        # restricted kinds of edit: the (r0 mod k)-th enabled kind
+        kinds = rnd.randint(1, 7)
+        got = oracle.mutate(s, *r, kinds=kinds, lib=lib)
+        assert list(got) == list_edit(s, *r, kinds=kinds), (s, r, kinds)
+    # moves only: a permutation of the sequence; hand cases with r0 arbitrary
+    assert list(oracle.mutate(seq, 0, 0, 3, kinds=4, lib=lib)) == [6, 7, 8, 5]
+    assert list(oracle.mutate(seq, 1, 3, 0, kinds=4, lib=lib)) == [8, 5, 6, 7]
+    assert list(oracle.mutate(seq, 1, 0, 0, kinds=5, lib=lib)) == [5, 6, 7, 8]   # insert|move, r0 = 1 -> move element 0 to index 0
+    assert list(oracle.mutate(seq, 2, 1, 0, kinds=3, lib=lib)) == [6, 5, 6, 7, 8]   # insert|delete, r0 = 2 -> insert
 
 
 def key_of(ev, M):
@@ -102,7 +112,7 @@ def _tiny_problem():
     return n, edges, w, m
 
 
-def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen, chain0=0):
+def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen, chain0=0, kinds=7):
     """The generation loop restated in Python over the separately pinned pieces, with the
     set-definition evaluator of defs.py in place of the oracle's evaluator."""
     def ev(s):
@@ -114,7 +124,7 @@ def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, ge
     for gen in range(gen0, gen0 + n_gen):
         for c, r in enumerate(rows):
             x = oracle.philox4x32_10([gen, chain0 + c, 0, 0], key, lib=lib)
-            child = list_edit(r, int(x[0]), int(x[1]), int(x[2]))
+            child = list_edit(r, int(x[0]), int(x[1]), int(x[2]), kinds)
             if child is None:
                 continue
             e = ev(child)
@@ -135,12 +145,13 @@ def pin_search_loop(make_graph, lib):
             seqs = np.array([x for r in rows for x in r], np.int32)
             lens = np.array([len(r) for r in rows], np.int32)
             chain0 = 0 if M == P0 else 1000
-            S = oracle.OracleSearch(g, seqs, lens, M, seed, chain0=chain0)
+            kinds = 7 if seed == 1 else (4 if M == 1 else 6)
+            S = oracle.OracleSearch(g, seqs, lens, M, seed, chain0=chain0, kinds=kinds)
             done = 0
             for n_gen in (1, 7, 40):
                 before = [key_of((S.peak[c], S.dur[c], S.status[c]), M) for c in range(S.P)]
                 S.run(n_gen)
-                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen, chain0)
+                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen, chain0, kinds)
                 done += n_gen
                 for c in range(S.P):
                     assert list(S.row(c)) == want_rows[c], (M, seed, c)

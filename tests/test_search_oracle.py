@@ -27,6 +27,7 @@ MUTANTS = {
                                        "child[j] = seq[j < T ? j : q]; child[j + (j < T)] = seq[q];\n        for (int32_t t = j + 1; t < T; ++t) child[t + 1] = seq[t];"),
     "insert_range_T": ("(r2 % ((uint32_t)T + 1u))", "(r2 % (uint32_t)T)"),
     "move_range_short": ("(int32_t)(r2 % (uint32_t)T); /* T = len + 1 insertion points */", "(int32_t)(r2 % (uint32_t)(T > 1 ? T - 1 : 1));"),
+    "kinds_mask_ignored": ("const uint32_t op = enabled[r0 % k];", "const uint32_t op = r0 % 3u;"),
     "ops_permuted": ("if (op == 1) return len;", "if (op == 2) return len;"),
     "accept_strict": ("return dur_c <= dur_p;", "return dur_c < dur_p;"),
     "accept_ignores_budget": ("const int64_t a = peak_c > M ? peak_c : M, b = peak_p > M ? peak_p : M;\n    if (a != b) return a < b;\n    return dur_c",
