@@ -176,7 +176,7 @@ int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t
  * Proposal of chain c in generation k for a sequence of T steps (T = 0 proposes nothing): with
  * (r0, r1, r2, r3) = Philox4x32-10(counter = (k, first_chain + c, 0, 0), key = (seed mod 2^32,
  * seed div 2^32)) (Salmon, Moraes, Dror, Shaw, SC 2011),
- *     op = r0 mod 3, q = r1 mod T;
+ *     op = r0 mod 3 (all kinds enabled, see moc_search_set_kinds), q = r1 mod T;
  *     op 0  insert: a further copy of node seq[q] is put in front of index j = r2 mod (T+1);
  *     op 1  delete: element q is removed;
  *     op 2  move:   element q is removed and put back in front of index j = r2 mod T of the
@@ -211,6 +211,19 @@ int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* le
  * plus one at the end, no allocation, no synchronisation).  Generations are numbered from 0 over
  * the life of the handle; the result does not depend on how they are split over calls. */
 int moc_search_run(moc_search* s, int32_t n_generations, void* stream);
+
+/*
+ * Chooses the kinds of edit the following generations may propose: bit 0 insert (MOC_EDIT_INSERT),
+ * bit 1 delete (MOC_EDIT_DELETE), bit 2 move (MOC_EDIT_MOVE); default all three.  With k kinds
+ * enabled a proposal takes the (r0 mod k)-th enabled kind in this order.  MOC_EDIT_MOVE alone
+ * searches over the orders of the sequences without adding or removing a copy: started from
+ * topological orders it is a search for a no-rematerialization order of low peak (Section 1: the
+ * peak depends on the topological order).  kinds outside 1..7 is MOC_ERR_ARG.
+ */
+#define MOC_EDIT_INSERT 1u
+#define MOC_EDIT_DELETE 2u
+#define MOC_EDIT_MOVE 4u
+int moc_search_set_kinds(moc_search* s, uint32_t kinds);
 
 /*
  * Copies the chains' current state to DEVICE arrays of the caller (any pointer may be NULL):

@@ -40,6 +40,8 @@ def load_library(path):
     lib.moc_oracle_graph_create.argtypes = [ctypes.c_int32, ctypes.c_int64, P, P, P, ctypes.c_int32]
     lib.moc_oracle_graph_destroy.restype = None
     lib.moc_oracle_graph_destroy.argtypes = [P]
+    lib.moc_oracle_graph_set_caps.restype = ctypes.c_int32
+    lib.moc_oracle_graph_set_caps.argtypes = [P, P]
     lib.moc_oracle_eval.restype = None
     lib.moc_oracle_eval.argtypes = [P, P, ctypes.c_int32, ctypes.c_int64, P, P, P, P, P]
     lib.moc_oracle_eval_batch.restype = ctypes.c_int32
@@ -91,6 +93,16 @@ class OracleGraph:
         if getattr(self, "_h", None):
             self._lib.moc_oracle_graph_destroy(self._h)
             self._h = None
+
+    def set_caps(self, caps):
+        """Per-node caps C_v in [1, C] (None: uniform C again)."""
+        if caps is None:
+            self._lib.moc_oracle_graph_set_caps(self._h, None)
+            return
+        caps = np.ascontiguousarray(caps, dtype=np.int32)
+        assert caps.shape == (self.n,)
+        if self._lib.moc_oracle_graph_set_caps(self._h, _ptr(caps)) != 0:
+            raise ValueError("oracle: cap outside [1, C]")
 
     def eval(self, seq, M):
         """One sequence -> dict(peak, dur, status, profile[T], free[T])."""

@@ -25,9 +25,9 @@
  *   memory     Eq. 4      : usage at step t = sum of m over the copies with s <= t <= e (both
  *                           ends inclusive); peak = maximum over the steps (Section 2).
  *   budget     Eq. 4      : feasible iff peak <= M.
- *   well-formedness       : every node at least once (Eq. 7), at most C copies of a node
- *                           (Section 2, parameter C_v, here uniform), hence n <= T <= C*n, ids in
- *                           range.
+ *   well-formedness       : every node at least once (Eq. 7), at most C_v copies of node v
+ *                           (Section 2, parameter C_v: uniform C unless per-node caps <= C are
+ *                           set), hence n <= T <= C*n, ids in range.
  *
  * Status codes: 1 feasible, 0 peak over budget, -1 a precedence constraint is violated
  * (peak = -1, duration still reported), -2 malformed sequence (peak = duration = -1).
@@ -49,6 +49,7 @@ typedef struct {
     int32_t *pred;       /* n_edges, grouped by consumer */
     uint8_t *has_succ;   /* n */
     int64_t *w, *m;      /* n */
+    int32_t *cap;        /* n per-node caps C_v, or NULL: every node may have C copies */
 } ograph;
 
 /* Builds the predecessor lists of G=(V,E) (Section 1: (u,v) in E, v needs the output of u). */
@@ -83,8 +84,22 @@ ograph *moc_oracle_graph_create(int32_t n, int64_t n_edges, const int32_t *edges
     return g;
 }
 
+/* Per-node caps C_v (Section 2: node v has at most C_v retention intervals), each in [1, C];
+ * NULL restores the uniform cap C.  Returns 0, or -1 for a cap outside [1, C]. */
+int32_t moc_oracle_graph_set_caps(ograph *g, const int32_t *caps) {
+    free(g->cap);
+    g->cap = NULL;
+    if (!caps) return 0;
+    for (int32_t v = 0; v < g->n; ++v)
+        if (caps[v] < 1 || caps[v] > g->C) return -1;
+    g->cap = (int32_t *)malloc((size_t)g->n * sizeof(int32_t));
+    memcpy(g->cap, caps, (size_t)g->n * sizeof(int32_t));
+    return 0;
+}
+
 void moc_oracle_graph_destroy(ograph *g) {
     if (!g) return;
+    free(g->cap);
     free(g->pred_start);
     free(g->pred);
     free(g->has_succ);
@@ -115,7 +130,7 @@ void moc_oracle_eval(const ograph *g, const int32_t *seq, int32_t T, int64_t M, 
         else count[seq[t]]++;
     }
     for (int32_t v = 0; v < n && ok; ++v)
-        if (count[v] < 1 || count[v] > g->C) ok = 0;
+        if (count[v] < 1 || count[v] > (g->cap ? g->cap[v] : g->C)) ok = 0;
     free(count);
     if (!ok) return;
 

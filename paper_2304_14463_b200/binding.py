@@ -20,7 +20,7 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
-           "moc_search_destroy"]
+           "moc_search_destroy", "moc_search_set_kinds"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -52,6 +52,8 @@ lib.moc_search_create.restype = ctypes.c_int
 lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, ctypes.c_uint32, _P, ctypes.POINTER(_P)]
 lib.moc_search_run.restype = ctypes.c_int
 lib.moc_search_run.argtypes = [_P, _i32, _P]
+lib.moc_search_set_kinds.restype = ctypes.c_int
+lib.moc_search_set_kinds.argtypes = [_P, ctypes.c_uint32]
 lib.moc_search_state.restype = ctypes.c_int
 lib.moc_search_state.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P]
 lib.moc_search_best.restype = ctypes.c_int
@@ -238,6 +240,13 @@ def moc_search_run(s, n_generations):
     _check(lib.moc_search_run(s, int(n_generations), _stream()), "moc_search_run")
 
 
+MOC_EDIT_INSERT, MOC_EDIT_DELETE, MOC_EDIT_MOVE = 1, 2, 4
+
+
+def moc_search_set_kinds(s, kinds):
+    _check(lib.moc_search_set_kinds(s, int(kinds)), "moc_search_set_kinds")
+
+
 def moc_search_info(s):
     P, stride, gen = _i32(), _i32(), ctypes.c_uint32()
     _check(lib.moc_search_info(s, ctypes.byref(P), ctypes.byref(stride), ctypes.byref(gen)), "moc_search_info")
@@ -346,6 +355,9 @@ class Search:
 
     def run(self, n_generations):
         moc_search_run(self.h, n_generations)
+
+    def set_kinds(self, kinds):
+        moc_search_set_kinds(self.h, kinds)
 
     def info(self):
         return moc_search_info(self.h)

@@ -76,6 +76,7 @@ int moc_search_create(const moc_graph* g, const int32_t* seqs, const int32_t* le
     p.seed_hi = (uint32_t)(seed >> 32);
     p.generation = 0;
     p.chain0 = first_chain;
+    p.kinds = 7u;
     p.rows = (int32_t*)(b + o_rows);
     p.c_offs = (int64_t*)(b + o_offs);
     p.peak = (int64_t*)(b + o_peak);
@@ -145,6 +146,13 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
     MOC_CUDA(cudaGetLastError());
     s->generation += (uint32_t)n_generations;
     launch_counter() = launches;
+    return MOC_OK;
+}
+
+int moc_search_set_kinds(moc_search* s, uint32_t kinds) {
+    clear_error();
+    if (!s || kinds == 0 || kinds > 7u) return fail(MOC_ERR_ARG, "moc_search_set_kinds: null handle or mask outside 1..7");
+    s->p.kinds = kinds;
     return MOC_OK;
 }
 

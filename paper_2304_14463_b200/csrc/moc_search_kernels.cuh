@@ -46,6 +46,7 @@ struct SearchParams {
     uint32_t seed_lo, seed_hi;
     uint32_t generation; // of the proposals written by this launch
     uint32_t chain0;     // global number of chain 0 (enters the random draws only)
+    uint32_t kinds;      // enabled kinds of edit: bit 0 insert, bit 1 delete, bit 2 move (never 0)
     int32_t* rows;       // 2 * P * stride
     int32_t* cur;        // P: 0 or 1
     int32_t* lens;       // P: length of each chain's sequence
@@ -74,7 +75,8 @@ constexpr int kSearchThreads = 256;  // 8 chains per block, one warp each
 
 // One warp per chain.  kSelect: settle the pending proposal of the chain (written by the previous
 // launch, scored since).  kPropose: write the next proposal.
-//   op = r0 mod 3 (0 insert, 1 delete, 2 move), q = r1 mod T the copy the edit refers to,
+//   op = the (r0 mod k)-th of the k enabled kinds in the order insert (0), delete (1), move (2); r0 mod 3
+//   when all are enabled; q = r1 mod T the copy the edit refers to,
 //   insert: the node seq[q] goes in front of index j = r2 mod (T+1);
 //   delete: element q is removed;
 //   move:   element q is removed and re-inserted in front of index j = r2 mod T of the shortened row.
@@ -115,7 +117,15 @@ __global__ void __launch_bounds__(kSearchThreads) search_step_kernel(const Searc
         return;
     }
     const uint4 r = philox4x32_10(make_uint4(p.generation, p.chain0 + (uint32_t)c, 0u, 0u), make_uint2(p.seed_lo, p.seed_hi));
-    const uint32_t op = r.x % 3u;
+    // the (r0 mod k)-th enabled kind, k = number of enabled kinds
+    const uint32_t nk = (uint32_t)__popc(p.kinds);
+    uint32_t pick = r.x % nk, op = 0;
+    for (uint32_t o = 0; o < 3; ++o) {
+        if (p.kinds >> o & 1u) {
+            if (pick == 0) { op = o; break; }
+            --pick;
+        }
+    }
     const int32_t q = (int32_t)(r.y % (uint32_t)T);
     // The proposal is "take element q out (delete, move), then put x in front of index j (insert,
     // move)"; qd / j beyond every index switch a half off.

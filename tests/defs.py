@@ -22,15 +22,15 @@ def succ_lists(n, edges):
     return succ, pred
 
 
-def set_definition(n, edges, w, m, C, seq, M):
-    """(status, peak, dur, profile) straight from the definitions; O(T^2)."""
+def set_definition(n, edges, w, m, C, seq, M, caps=None):
+    """(status, peak, dur, profile) straight from the definitions; O(T^2).  caps: per-node C_v."""
     T = len(seq)
     succ, pred = succ_lists(n, edges)
     if T < n or T > C * n or any(v < 0 or v >= n for v in seq):
         return -2, -1, -1, None
     for v in range(n):
         k = sum(1 for x in seq if x == v)
-        if k < 1 or k > C:
+        if k < 1 or k > (C if caps is None else caps[v]):
             return -2, -1, -1, None
     dur = sum(w[v] for v in seq)
     # Eq. 5: each consumer needs an earlier copy of every predecessor

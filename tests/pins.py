@@ -163,6 +163,39 @@ def pin_exhaustive(make_graph):
                     assert list(r["profile"]) == prof, (n, edges, seq)
 
 
+def pin_node_caps(make_graph):
+    """Per-node caps C_v (Section 2): hand cases on the paper's 4-node graph, then every sequence up
+    to length 6 on two small graphs against the set definition with the same caps."""
+    n, edges = 4, [(0, 1), (1, 2), (2, 3), (0, 3)]
+    G = make_graph(n, edges, [2, 3, 4, 5], [1, 1, 1, 1], 2)
+    seq = [0, 1, 2, 0, 3]
+    base = G.eval(seq, BIG)
+    assert base["status"] == 1 and base["peak"] == 3
+    G.set_caps([1, 2, 2, 2])                      # node 0 may not be recomputed
+    r = G.eval(seq, BIG)
+    assert (r["status"], r["peak"], r["dur"]) == (-2, -1, -1)
+    assert G.eval([0, 1, 2, 3], BIG)["status"] == 1
+    G.set_caps([2, 1, 1, 1])                      # only node 0 may be: unchanged result
+    r = G.eval(seq, BIG)
+    assert (r["status"], r["peak"], r["dur"]) == (1, 3, 16) and list(r["profile"]) == list(base["profile"])
+    assert G.eval([0, 1, 1, 2, 3], BIG)["status"] == -2
+    G.set_caps(None)                              # uniform cap again
+    assert G.eval([0, 1, 1, 2, 3], BIG)["status"] == 1
+    rnd = random.Random(5)
+    for n, edges, caps in [(4, [(0, 1), (0, 2), (1, 3), (2, 3)], [1, 3, 2, 1]), (3, [(0, 1), (1, 2)], [3, 1, 2])]:
+        m = [rnd.randint(1, 20) for _ in range(n)]
+        w = [rnd.randint(1, 9) for _ in range(n)]
+        M = sum(m) * 2 // 3
+        G = make_graph(n, edges, w, m, 3)
+        G.set_caps(caps)
+        for T in range(n, 7):
+            for seq in itertools.product(range(n), repeat=T):
+                seq = list(seq)
+                st, peak, dur, prof = defs.set_definition(n, edges, w, m, 3, seq, M, caps=caps)
+                r = G.eval(seq, M)
+                assert (r["status"], r["peak"], r["dur"]) == (st, peak, dur), (n, edges, caps, seq)
+
+
 def _random_remat_seq(rnd, n, edges, C, p):
     order = rnd.choice(list(itertools.islice(defs.topological_orders(n, edges), 50)))
     seq = list(order)
@@ -213,7 +246,7 @@ def pin_random_remat(make_graph, n_cases=150):
 
 
 ALL_PINS = [pin_paper_example, pin_chain, pin_small_cases, pin_topological_orders, pin_exhaustive,
-            pin_random_remat]
+            pin_random_remat, pin_node_caps]
 
 
 def run_all(make_graph):

@@ -129,3 +129,26 @@ def test_search_split_invariance_and_errors(B):
     bad = np.zeros(4 * wl.n, np.int32)
     s = B.Search(G, dev(bad), dev(np.full(4, wl.n, np.int32)), M, 1)
     assert s.best()["index"] == -1
+
+
+@pytest.mark.parametrize("kinds", [4, 3, 5, 6, 1, 2])
+def test_search_restricted_kinds(B, kinds):
+    """Masks of enabled edits; moves only keeps every length and searches over orders."""
+    wl = W.make(1, seed=2, B=256)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    S = B.Search(G, dev(wl.seqs), dev(wl.lens), M, 21)
+    S.set_kinds(kinds)
+    OS = OracleSearch(O, wl.seqs, wl.lens, M, 21, stride=S.info()["stride"], kinds=kinds)
+    for g in (3, 30):
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"kinds {kinds} after {OS.generation}")
+    if kinds == 4:
+        assert (OS.lens == wl.lens).all()
+    with pytest.raises(B.MocError):
+        S.set_kinds(0)
+    with pytest.raises(B.MocError):
+        S.set_kinds(8)

@@ -32,7 +32,9 @@ MUTANTS = {
     # allocation one step late
     "alloc_late": ("delta[p] += g->m[seq[p]];", "delta[p + 1] += g->m[seq[p]];"),
     # copy-count cap ignored
-    "no_cap": ("if (count[v] < 1 || count[v] > g->C) ok = 0;", "if (count[v] < 1) ok = 0;"),
+    "no_cap": ("if (count[v] < 1 || count[v] > (g->cap ? g->cap[v] : g->C)) ok = 0;", "if (count[v] < 1) ok = 0;"),
+    # per-node caps ignored
+    "node_caps_ignored": ("count[v] > (g->cap ? g->cap[v] : g->C)", "count[v] > g->C"),
     # wrong weight array in the profile
     "w_for_m": ("delta[p] += g->m[seq[p]];\n        delta[fr[p] + 1] -= g->m[seq[p]];",
                 "delta[p] += g->w[seq[p]];\n        delta[fr[p] + 1] -= g->w[seq[p]];"),
