@@ -74,8 +74,18 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                      const int64_t* m, moc_graph** out);
 
 /* Sets the cap C on copies per node (the paper's C_v, uniform over nodes; Section 2).
- * 1 <= C <= MOC_MAX_COPIES, else MOC_ERR_ARG. */
+ * 1 <= C <= MOC_MAX_COPIES, else MOC_ERR_ARG.  Per-node caps set earlier are dropped. */
 int moc_graph_set_max_copies(moc_graph* g, int32_t C);
+
+/*
+ * Per-node caps C_v (Section 2: node v has at most C_v retention intervals).
+ *   caps   HOST, n ints, each in [1, C] for the handle's current C; NULL restores the uniform cap.
+ * A sequence with more than C_v copies of node v gets status -2.  The length bound stays
+ * n <= T <= C*n.  moc_graph_set_max_copies resets the caps to uniform.  Synchronises the device
+ * (work in flight may still read the old caps), then copies.  Errors: MOC_ERR_ARG, MOC_ERR_CUDA,
+ * MOC_ERR_NOMEM.
+ */
+int moc_graph_set_node_caps(moc_graph* g, const int32_t* caps);
 
 /* Frees the handle with its device memory.  NULL is accepted.  The caller must have
  * synchronised every stream that still runs work of this handle. */

@@ -20,7 +20,7 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
-           "moc_search_destroy", "moc_search_set_kinds"]
+           "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -32,6 +32,8 @@ lib.moc_graph_create.restype = ctypes.c_int
 lib.moc_graph_create.argtypes = [_i32, _i64, _P, _P, _P, ctypes.POINTER(_P)]
 lib.moc_graph_set_max_copies.restype = ctypes.c_int
 lib.moc_graph_set_max_copies.argtypes = [_P, _i32]
+lib.moc_graph_set_node_caps.restype = ctypes.c_int
+lib.moc_graph_set_node_caps.argtypes = [_P, _P]
 lib.moc_graph_destroy.restype = None
 lib.moc_graph_destroy.argtypes = [_P]
 lib.moc_graph_info.restype = ctypes.c_int
@@ -133,6 +135,16 @@ def moc_graph_create(n, edges, w, m):
 
 def moc_graph_set_max_copies(g, C):
     _check(lib.moc_graph_set_max_copies(g, int(C)), "moc_graph_set_max_copies")
+
+
+def moc_graph_set_node_caps(g, caps):
+    """caps: n ints (host), each in [1, C]; None restores the uniform cap."""
+    import numpy as np
+    if caps is None:
+        _check(lib.moc_graph_set_node_caps(g, None), "moc_graph_set_node_caps")
+        return
+    caps = np.ascontiguousarray(caps, np.int32)
+    _check(lib.moc_graph_set_node_caps(g, caps.ctypes.data), "moc_graph_set_node_caps")
 
 
 def moc_graph_set_launch(g, threads_per_sequence=0, sequences_per_block=0):
@@ -309,6 +321,11 @@ class Graph:
 
     def info(self):
         return moc_graph_info(self.h)
+
+    def set_caps(self, caps):
+        if caps is not None and len(caps) != self.n:
+            raise ValueError("caps must have n entries")
+        moc_graph_set_node_caps(self.h, caps)
 
     def set_timing_events(self, before=None, after=None):
         moc_graph_set_timing_events(self.h, before, after)

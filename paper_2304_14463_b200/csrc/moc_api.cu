@@ -226,6 +226,7 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     p.g.succ = g->d_succ;
     p.g.w = g->d_w;
     p.g.m = pl.wide ? (const void*)g->d_m64 : (const void*)g->d_m32;
+    p.g.cap = g->d_cap;
     p.cnt_bytes = pl.cnt_bytes;
     p.occ_bytes = pl.occ_bytes;
     p.delta_bytes = pl.delta_bytes;
@@ -403,6 +404,12 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
 
     moc_graph* g = new (std::nothrow) moc_graph();
     if (!g) return fail(MOC_ERR_NOMEM, "host allocation failed");
+    try {
+        g->h_w.assign(w, w + n);
+    } catch (const std::bad_alloc&) {
+        delete g;
+        return fail(MOC_ERR_NOMEM, "host allocation failed");
+    }
     g->n = n;
     g->n_edges = ne;
     g->sum_m = sum_m;
@@ -506,6 +513,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                     pos += 32 * (uint32_t)rows[d];
                 }
                 g->sell_len = (int32_t)sell_len;
+                g->h_slot = slot;
                 g->n_tiles = n_tiles;
                 up(&g->d_rec32, rec32.data(), rec32.size() * sizeof(rec32[0]));
                 up(&g->d_rec64, rec64.data(), rec64.size() * sizeof(rec64[0]));
@@ -532,10 +540,57 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
 int moc_graph_set_max_copies(moc_graph* g, int32_t C) {
     g_err[0] = 0;
     if (!g || C < 1 || C > MOC_MAX_COPIES) return fail(MOC_ERR_ARG, "moc_graph_set_max_copies: C must be 1..%d", MOC_MAX_COPIES);
+    if (!g->h_cap.empty()) {   // caps refer to the old C: back to a uniform cap
+        int rc = moc_graph_set_node_caps(g, nullptr);
+        if (rc != MOC_OK) return rc;
+    }
     g->C = C;
     g->plan_eval.valid = false;
     g->plan_profile.valid = false;
     return MOC_OK;
+}
+
+// Uploads the slot durations of the warp-per-sequence layout, with bit 63 marking nodes whose cap is 1.
+static int upload_wslot(moc_graph* g) {
+    if (!g->d_wslot) return MOC_OK;
+    std::vector<int64_t> wslot(g->h_slot.size());
+    for (size_t r = 0; r < wslot.size(); ++r) {
+        const int32_t v = g->h_slot[r];
+        int64_t x = v >= 0 ? g->h_w[v] : 0;
+        if (v >= 0 && !g->h_cap.empty() && g->h_cap[v] == 1) x |= INT64_MIN;
+        wslot[r] = x;
+    }
+    MOC_CUDA(cudaMemcpy(g->d_wslot, wslot.data(), wslot.size() * 8, cudaMemcpyHostToDevice));
+    return MOC_OK;
+}
+
+int moc_graph_set_node_caps(moc_graph* g, const int32_t* caps) {
+    g_err[0] = 0;
+    if (!g) return fail(MOC_ERR_ARG, "moc_graph_set_node_caps: null handle");
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    // work queued on any stream may still read the old caps
+    MOC_CUDA(cudaDeviceSynchronize());
+    try {
+        if (!caps) {
+            g->h_cap.clear();
+        } else {
+            for (int32_t v = 0; v < g->n; ++v)
+                if (caps[v] < 1 || caps[v] > g->C)
+                    return fail(MOC_ERR_ARG, "moc_graph_set_node_caps: cap %d of node %d outside [1, C = %d]", caps[v], v, g->C);
+            g->h_cap.assign(caps, caps + g->n);
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(MOC_ERR_NOMEM, "host allocation failed");
+    }
+    if (caps) {
+        if (!g->d_cap) MOC_CUDA(cudaMalloc((void**)&g->d_cap, std::max<size_t>((size_t)g->n * 4, 16)));
+        MOC_CUDA(cudaMemcpy(g->d_cap, caps, (size_t)g->n * 4, cudaMemcpyHostToDevice));
+    } else if (g->d_cap) {
+        MOC_CUDA(cudaFree(g->d_cap));
+        g->d_cap = nullptr;
+    }
+    return upload_wslot(g);
 }
 
 int moc_graph_set_launch(moc_graph* g, int32_t tps, int32_t spb) {
@@ -569,6 +624,7 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_rec32);
     cudaFree(g->d_rec64);
     cudaFree(g->d_wslot);
+    cudaFree(g->d_cap);
     cudaFree(g->d_sell);
     cudaFree(g->d_tile);
     cudaFree(g->d_offs);

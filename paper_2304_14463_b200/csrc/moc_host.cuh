@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/moc.h"
 #include "moc_kernels.cuh"
 #include "moc_pair_kernel.cuh"
@@ -78,6 +80,10 @@ struct moc_graph {
     void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
     void* d_rec64 = nullptr;
     int64_t* d_wslot = nullptr;
+    int32_t* d_cap = nullptr;             // per-node caps C_v, or null: uniform C
+    std::vector<int32_t> h_slot;          // node of every slot of the warp-per-sequence layout (-1: none)
+    std::vector<int64_t> h_w;             // durations (host copy, to rebuild d_wslot)
+    std::vector<int32_t> h_cap;           // per-node caps (empty: uniform)
     uint32_t* d_sell = nullptr;
     uint32_t* d_tile = nullptr;
     // grow-only scratch; mutable because evaluation takes a const handle

@@ -28,6 +28,7 @@ struct GraphDev {
     const int32_t* succ;        // distinct edges, grouped by producer
     const int64_t* w;           // n durations
     const void* m;              // n output sizes, int32 or int64 (matches MemT)
+    const int32_t* cap;         // n per-node caps C_v <= C, or nullptr: every node may have C copies
 };
 
 struct EvalParams {
@@ -181,6 +182,7 @@ __device__ __forceinline__ void eval_one(const EvalParams& p, const int b, const
         for (int u = tid; u < n; u += G) {
             const int c = cnt[u];
             if (c < 1) bad = 1;
+            if (p.g.cap != nullptr && c > __ldg(&p.g.cap[u])) bad = 1;
             uint32_t o[CP], f[CP];
 #pragma unroll
             for (int j = 0; j < CP; ++j) o[j] = occ[u * CP + j];

@@ -48,7 +48,7 @@ struct PairParams {
     int32_t max_T;             // C * n
     uint32_t sum_bias;         // number of empty node slots (each reads a word holding (1, 1))
     const void* rec;           // 64 * n_tiles node records (NodeRec<MemT>), slot = half * 32 + lane
-    const int64_t* wslot;      // 64 * n_tiles durations, same slots
+    const int64_t* wslot;      // 64 * n_tiles durations, same slots; bit 63 set: the node's cap C_v is 1
     const uint32_t* sell;      // sell_len entries: successor word offsets of the two halves, 16 bits each
     const uint32_t* tile;      // n_tiles: first entry of the tile | rows of the tile << 20
     int64_t base_dur;          // sum of all w
@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(kPre > 0 ? 384 : 512, kPre > 0 ? 2 : 1) eval_p
 
             // ---- stage 2 and the scatter of stage 3: two node slots per lane and tile
             uint32_t vmin = 0xFFFFFFFFu, vsum = 0;
-            uint32_t depw = 0;
+            uint32_t depw = 0, capw = 0;
             int64_t dur_extra = 0;
             for (int d = 0; d < p.n_tiles; ++d) {
                 Rec rec[2];
@@ -349,7 +349,11 @@ __global__ void __launch_bounds__(kPre > 0 ? 384 : 512, kPre > 0 ? 2 : 1) eval_p
                     red_add_shared(da + (fb << kShift), (MemT)(-rec[h].m));
                     if (a != bpos) {
                         vsum += a;
-                        dur_extra += s_w[(2 * d + h) * 32 + lane];
+                        // bit 63 of the duration marks a node that may have one copy only (C_v = 1): the
+                        // sequence is then malformed and the sum below is never reported
+                        const int64_t wv = s_w[(2 * d + h) * 32 + lane];
+                        capw |= (uint32_t)((uint64_t)wv >> 32);
+                        dur_extra += wv;
                         // latest successor copy x with a < x < b, if any: (x - b) mod 2^16 is the largest
                         const uint32_t x = (max_u16x2(G[h], swap_halves(G[h])) + bpos) & 0xFFFFu;
                         const uint32_t fa = (x - 1u < bpos - 1u) ? x : a;
@@ -360,7 +364,8 @@ __global__ void __launch_bounds__(kPre > 0 ? 384 : 512, kPre > 0 ? 2 : 1) eval_p
             }
             vmin = __reduce_min_sync(0xFFFFFFFFu, vmin);
             vsum = __reduce_add_sync(0xFFFFFFFFu, vsum);
-            const bool well_formed = vmin != 0 && vsum == (uint32_t)T * ((uint32_t)T + 1u) / 2u + p.sum_bias;
+            const bool cap_ok = !__any_sync(0xFFFFFFFFu, (int32_t)capw < 0);
+            const bool well_formed = cap_ok && vmin != 0 && vsum == (uint32_t)T * ((uint32_t)T + 1u) / 2u + p.sum_bias;
             const bool dep = __any_sync(0xFFFFFFFFu, depw != 0);
             __syncwarp();
 

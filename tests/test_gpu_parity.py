@@ -45,6 +45,9 @@ def test_pins_through_the_gpu(B):
         def __init__(self, n, edges, w, m, C):
             self.G = B.Graph(n, edges, w, m, C)
 
+        def set_caps(self, caps):
+            self.G.set_caps(caps)
+
         def eval(self, seq, M):
             seq = np.asarray(seq, np.int32)
             p, d, s = gpu_eval(self.G, seq, np.array([len(seq)], np.int32), M)
@@ -54,7 +57,7 @@ def test_pins_through_the_gpu(B):
             return dict(peak=int(p[0]), dur=int(d[0]), status=int(s[0]),
                         profile=prof.cpu().numpy(), free=free.cpu().numpy())
 
-    for pin in (pins.pin_paper_example, pins.pin_small_cases, pins.pin_random_remat):
+    for pin in (pins.pin_paper_example, pins.pin_small_cases, pins.pin_random_remat, pins.pin_node_caps):
         pin(lambda n, e, w, m, C: GpuGraph(n, e, w, m, C))
 
 
@@ -329,3 +332,26 @@ def test_sampled_invariants_at_full_size(B):
     wsum = np.add.reduceat(wl.w[wl.seqs], offs[:-1])
     msum = np.add.reduceat(wl.m[wl.seqs], offs[:-1])
     assert (dur == wsum).all() and (peak <= msum).all()
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_node_caps_parity(B, idx):
+    """Random per-node caps C_v on the warp-per-sequence kernel (C = 2) and the group kernel (C = 3)."""
+    wl = W.make(idx, seed=2, B=[0, 2048, 1024, 256][idx])
+    rng = np.random.default_rng(idx)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=4, frac=1 / 16)
+    M = O.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    for frac_one in (0.02, 0.5, 1.0):
+        caps = np.where(rng.random(wl.n) < frac_one, 1, rng.integers(1, wl.C + 1, wl.n)).astype(np.int32)
+        O.set_caps(caps)
+        G.set_caps(caps)
+        _, _, st = assert_batch_equal(G, O, seqs, lens, M, f"caps {frac_one}")
+        assert (st == -2).any()
+    O.set_caps(None)
+    G.set_caps(None)
+    _, _, st = assert_batch_equal(G, O, seqs, lens, M, "caps cleared")
+    assert (st >= 0).any()
+    with pytest.raises(B.MocError):
+        G.set_caps(np.full(wl.n, wl.C + 1, np.int32))
