@@ -36,6 +36,8 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the evaluation kernel, from
 # one ncu capture with flushed caches (None when the kernel changed after the capture)
 NCU_TRAFFIC_BYTES = 34865920
+# executed warp instructions of the same launch (smsp__inst_executed.sum of that capture)
+NCU_WARP_INSTRUCTIONS = 32496634
 NCU_TRAFFIC_SOURCE = "ncu --set full, one launch: dram read 34.86 MB, write 0 (the 0.33 MB of results were still in L2)"
 
 
@@ -409,6 +411,16 @@ def main():
                                  "not by HBM (ncu: issue slots 65 %, ALU pipe 55 %, shared-memory data pipe 64 %, DRAM 9 % busy)"},
             "clocks": clocks.summary(),
         }
+        if args.workload == WORKLOAD_IDX:
+            # Second view of the same launch: the limit ncu shows is instruction issue and the integer /
+            # shared-memory pipes.  Issue peak = SMs x 4 schedulers x 1 warp instruction per clock.
+            sm_mhz = line["clocks"]["sm_mhz"] or 1965.0
+            issue_peak = 148 * 4 * sm_mhz * 1e6
+            line["issue_roofline"] = {"bound": "alu", "achieved": NCU_WARP_INSTRUCTIONS / (kernel_ms * 1e-3) / 1e9,
+                                      "peak": issue_peak / 1e9, "unit": "G warp instructions/s",
+                                      "frac": NCU_WARP_INSTRUCTIONS / (kernel_ms * 1e-3) / issue_peak,
+                                      "note": "executed (not algorithmic) instructions of one launch from the ncu capture; "
+                                              "context for the HBM fraction above, not a replacement"}
         if not args.no_cpu_baseline:
             o = time_oracle(base, M)
             res = o["all"][3]
