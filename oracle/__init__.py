@@ -16,18 +16,20 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "moc_oracle.c")
 _SRC_SEARCH = os.path.join(_HERE, "moc_search_oracle.c")
+_SRC_INTERVAL = os.path.join(_HERE, "moc_interval_oracle.c")
+_HDR = os.path.join(_HERE, "moc_oracle_graph.h")
 _LIB = os.path.join(_HERE, "libmoc_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
-    """Compiles moc_oracle.c and moc_search_oracle.c into libmoc_oracle.so next to them (gcc -O2);
+    """Compiles moc_oracle.c and moc_search_oracle.c and moc_interval_oracle.c into libmoc_oracle.so next to them (gcc -O2);
     returns the path."""
-    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_SEARCH))
+    newest = max(os.path.getmtime(f) for f in (_SRC, _SRC_SEARCH, _SRC_INTERVAL, _HDR))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".{os.getpid()}.tmp"
         subprocess.run(["gcc", "-O2", "-std=c11", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC,
-                        _SRC_SEARCH], check=True)
+                        _SRC_SEARCH, _SRC_INTERVAL], check=True)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -47,6 +49,11 @@ def load_library(path):
     lib.moc_oracle_eval_batch.restype = ctypes.c_int32
     lib.moc_oracle_eval_batch.argtypes = [P, P, P, ctypes.c_int64, ctypes.c_int64, P, P, P,
                                           ctypes.c_int32]
+    if hasattr(lib, "moc_oracle_check_intervals"):
+        lib.moc_oracle_check_intervals.restype = None
+        lib.moc_oracle_check_intervals.argtypes = [P, P, P, P, ctypes.c_int64, P, ctypes.c_int64, P, P, P, P]
+        lib.moc_oracle_intervals_to_sequence.restype = ctypes.c_int32
+        lib.moc_oracle_intervals_to_sequence.argtypes = [P, P, P, P, ctypes.c_int64, P]
     if hasattr(lib, "moc_oracle_search_run"):
         u32, u64, i32, i64 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_int64
         lib.moc_oracle_philox4x32_10.restype = None
@@ -117,6 +124,34 @@ class OracleGraph:
                                 _ptr(profile), _ptr(free))
         return dict(peak=int(peak[0]), dur=int(dur[0]), status=int(status[0]),
                     profile=profile[:T].copy(), free=free[:T].copy())
+
+    def check_intervals(self, s, e, a, M, D=None, topo_index=None):
+        """One solution in interval form ([n, C] int32 arrays s, e, a) -> dict(mask, peak, dur).
+        topo_index (1-based index of every node in the input topological order) selects the staged
+        model; D defaults to C*n (plain) or n(n+1)/2 (staged)."""
+        s = np.ascontiguousarray(s, dtype=np.int32).reshape(self.n, self.C)
+        e = np.ascontiguousarray(e, dtype=np.int32).reshape(self.n, self.C)
+        a = np.ascontiguousarray(a, dtype=np.int32).reshape(self.n, self.C)
+        ti = None if topo_index is None else np.ascontiguousarray(topo_index, dtype=np.int32)
+        if D is None:
+            D = self.C * self.n if ti is None else self.n * (self.n + 1) // 2
+        peak, dur, mask = np.zeros(1, np.int64), np.zeros(1, np.int64), np.zeros(1, np.int32)
+        usage = np.full(int(D), -1, np.int64)
+        self._lib.moc_oracle_check_intervals(self._h, _ptr(s), _ptr(e), _ptr(a), int(D),
+                                             None if ti is None else _ptr(ti), int(M), _ptr(peak), _ptr(dur), _ptr(mask),
+                                             _ptr(usage))
+        return dict(mask=int(mask[0]), peak=int(peak[0]), dur=int(dur[0]), usage=usage)
+
+    def intervals_to_sequence(self, s, e, a, D=None, staged=False):
+        """Execution sequence of a solution in interval form, or None when it has none."""
+        s = np.ascontiguousarray(s, dtype=np.int32).reshape(self.n, self.C)
+        e = np.ascontiguousarray(e, dtype=np.int32).reshape(self.n, self.C)
+        a = np.ascontiguousarray(a, dtype=np.int32).reshape(self.n, self.C)
+        if D is None:
+            D = self.n * (self.n + 1) // 2 if staged else self.C * self.n
+        out = np.zeros(self.n * self.C, np.int32)
+        k = self._lib.moc_oracle_intervals_to_sequence(self._h, _ptr(s), _ptr(e), _ptr(a), int(D), _ptr(out))
+        return None if k < 0 else out[:k].copy()
 
     def eval_batch(self, seqs, lens, M, n_threads=1):
         """Packed batch -> (peak[B], dur[B], status[B], threads_used)."""

@@ -41,16 +41,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-typedef struct {
-    int32_t n;
-    int32_t C;
-    int64_t n_edges;
-    int64_t *pred_start; /* n+1 */
-    int32_t *pred;       /* n_edges, grouped by consumer */
-    uint8_t *has_succ;   /* n */
-    int64_t *w, *m;      /* n */
-    int32_t *cap;        /* n per-node caps C_v, or NULL: every node may have C copies */
-} ograph;
+#include "moc_oracle_graph.h"
 
 /* Builds the predecessor lists of G=(V,E) (Section 1: (u,v) in E, v needs the output of u). */
 ograph *moc_oracle_graph_create(int32_t n, int64_t n_edges, const int32_t *edges, const int64_t *w,

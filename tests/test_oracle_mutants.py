@@ -57,7 +57,7 @@ def test_mutant_is_caught(name, tmp_path):
     c = tmp_path / "mutant.c"
     so = tmp_path / "mutant.so"
     c.write_text(mutated)
-    subprocess.run(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-pthread", "-o", str(so), str(c)], check=True)
+    subprocess.run(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-pthread", "-I", os.path.dirname(SRC), "-o", str(so), str(c)], check=True)
     lib = oracle.load_library(str(so))
 
     def make_graph(n, edges, w, m, C):

@@ -49,7 +49,7 @@ def test_search_mutant_is_caught(name, tmp_path):
     c = tmp_path / "mutant.c"
     so = tmp_path / "mutant.so"
     c.write_text(src.replace(old, new))
-    subprocess.run(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-pthread", "-o", str(so), str(c), SRC_EVAL], check=True)
+    subprocess.run(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-pthread", "-I", os.path.dirname(SRC), "-o", str(so), str(c), SRC_EVAL], check=True)
     lib = oracle.load_library(str(so))
     with pytest.raises(AssertionError):
         search_pins.run_all(lambda n, e, w, m, C: oracle.OracleGraph(n, e, w, m, C, lib=lib), lib)
