@@ -170,6 +170,45 @@ int moc_mem_profile(const moc_graph* g, const int32_t* seq, int32_t len, int64_t
                     int32_t* out_free, int32_t* out_status, void* stream);
 
 /*
+ * ---- Solutions in the paper's own variables ------------------------------------------------------
+ *
+ * Checks B solutions given as retention intervals against Eqs. 2-8 as printed (Section 2), with the
+ * duration of Eq. 1 and the peak of the usage of Eq. 4, e.g. to validate what a constraint solver
+ * returned.  Node v has C slots (the handle's C); slot i has a start s, an end e (events, 1-based)
+ * and a flag a (1 active, 0 inactive).
+ *   s, e, a      DEVICE, B*n*C int32 each, index [b][v][i].
+ *   D            size of the event domain {1..D}: normally C*n (Section 2) or n(n+1)/2 (staged).
+ *   topo_index   DEVICE, n int32: 1-based index of every node in the input topological order; selects
+ *                the staged model of the subsection "Complexity Reduction by Enforcing an Initial
+ *                Topological Ordering" (stage j = events j(j-1)/2+1 .. j(j+1)/2; an active interval of
+ *                the node with index k starts at event k of a stage j >= k; its first interval at the
+ *                last event of stage k).  Requires D = n(n+1)/2.  NULL: the plain model.
+ *   M            memory budget of Eq. 4.
+ *   out_mask     DEVICE, B int32: bit 0 set when Eq. 2 (s <= e, every slot) is violated, bit 1 Eq. 3
+ *                (e_v^i <= s_v^{i+1}, every slot), bit 2 Eq. 4 (peak > M), bit 3 Eq. 5 (an active
+ *                interval of a consumer v starts at t without an active interval of a predecessor u
+ *                with s_u + 1 <= t <= e_u), bit 4 Eq. 6 (two slots of different nodes share a start;
+ *                plain model only), bit 5 Eq. 7 (first slot inactive), bit 6 Eq. 8 (s or e outside
+ *                {1..D}, a outside {0,1}), bit 7 the staged rule.  When bit 6 is set nothing else is
+ *                evaluated: mask = 64, peak = duration = -1, length = -1.
+ *   out_peak     DEVICE, B int64: max over the events of the sum of m over active intervals with
+ *                s <= t <= e.
+ *   out_dur      DEVICE, B int64: sum of w over active intervals.
+ *   out_seqs     DEVICE, B rows of n*C int32, or NULL: the execution sequence the solution stands for
+ *                (its active intervals in the order of their starts), usable with moc_eval_batch after
+ *                packing; only the first out_lens[b] entries of a row are written.
+ *   out_lens     DEVICE, B int32, or NULL: number of active intervals, or -1 when two of them start at
+ *                the same event (no sequential execution; the row is then left untouched).
+ * Asynchronous on `stream`; allocates nothing.  MOC_ERR_ARG when the domain and the intervals of one
+ * solution do not fit in the shared memory of one block ((D/32)*12 + n*C*8 bytes, roughly).
+ * Per-node caps of the handle are not applied here: every node has the handle's C slots.
+ */
+int moc_check_intervals(const moc_graph* g, const int32_t* s, const int32_t* e, const int32_t* a,
+                        int32_t B, int64_t D, const int32_t* topo_index, int64_t M, int64_t* out_peak,
+                        int64_t* out_dur, int32_t* out_mask, int32_t* out_seqs, int32_t* out_lens,
+                        void* stream);
+
+/*
  * ---- Local search over sequences (Section 3, "Optimization in Two Phases") -------------------------
  *
  * P independent chains each hold one sequence and its evaluation.  One generation proposes, for

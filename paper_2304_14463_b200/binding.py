@@ -20,7 +20,7 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
-           "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps"]
+           "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -50,6 +50,8 @@ lib.moc_graph_set_launch.restype = ctypes.c_int
 lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
 lib.moc_graph_set_timing_events.restype = ctypes.c_int
 lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
+lib.moc_check_intervals.restype = ctypes.c_int
+lib.moc_check_intervals.argtypes = [_P, _P, _P, _P, _i32, _i64, _P, _i64, _P, _P, _P, _P, _P, _P]
 lib.moc_search_create.restype = ctypes.c_int
 lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, ctypes.c_uint32, _P, ctypes.POINTER(_P)]
 lib.moc_search_run.restype = ctypes.c_int
@@ -237,6 +239,26 @@ def moc_last_launch_count():
     return lib.moc_last_launch_count()
 
 
+def moc_check_intervals(g, s, e, a, M, D, topo_index=None, want_seqs=True):
+    """Device tensors s, e, a of shape [B, n, C] (int32) -> dict of device tensors mask, peak, dur and,
+    with want_seqs, seqs [B, n*C] and lens."""
+    import torch
+    B, K = s.shape[0], s.shape[1] * s.shape[2]
+    peak = torch.empty(B, dtype=torch.int64, device=s.device)
+    dur = torch.empty(B, dtype=torch.int64, device=s.device)
+    mask = torch.empty(B, dtype=torch.int32, device=s.device)
+    seqs = torch.full((B, K), -1, dtype=torch.int32, device=s.device) if want_seqs else None
+    lens = torch.empty(B, dtype=torch.int32, device=s.device) if want_seqs else None
+    rc = lib.moc_check_intervals(g, _dev(s, torch.int32, "s"), _dev(e, torch.int32, "e"), _dev(a, torch.int32, "a"),
+                                 B, int(D), _dev(topo_index, torch.int32, "topo_index") if topo_index is not None else None,
+                                 int(M), _dev(peak, torch.int64, "peak"), _dev(dur, torch.int64, "dur"),
+                                 _dev(mask, torch.int32, "mask"),
+                                 _dev(seqs, torch.int32, "seqs") if want_seqs else None,
+                                 _dev(lens, torch.int32, "lens") if want_seqs else None, _stream())
+    _check(rc, "moc_check_intervals")
+    return dict(mask=mask, peak=peak, dur=dur, seqs=seqs, lens=lens)
+
+
 def moc_search_create(g, seqs, lens, M, seed, first_chain=0):
     """Device tensors (packed sequences, lengths) -> search handle; synchronous."""
     import torch
@@ -341,6 +363,11 @@ class Graph:
 
     def mem_profile(self, seq, want_free=True):
         return moc_mem_profile(self.h, seq, want_free)
+
+    def check_intervals(self, s, e, a, M, D=None, topo_index=None, want_seqs=True):
+        if D is None:
+            D = self.n * (self.n + 1) // 2 if topo_index is not None else self.C * self.n
+        return moc_check_intervals(self.h, s, e, a, M, D, topo_index, want_seqs)
 
     def no_remat_peak(self):
         """Peak of the identity order 0..n-1 (the input topological order when ids are topological),
