@@ -17,6 +17,7 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
     if (!s || !e || !a || !out_peak || !out_dur || !out_mask)
         return fail(MOC_ERR_ARG, "moc_check_intervals: null array");
     if (D < 1 || D > ((int64_t)1 << 30)) return fail(MOC_ERR_ARG, "moc_check_intervals: D outside [1, 2^30]");
+    if (g->C > moc::kIvMaxC) return fail(MOC_ERR_ARG, "moc_check_intervals: C > %d", moc::kIvMaxC);
     const int64_t n = g->n, K = n * g->C;
     if (topo_index && D != n * (n + 1) / 2)
         return fail(MOC_ERR_ARG, "moc_check_intervals: the staged model needs D = n(n+1)/2 = %lld", (long long)(n * (n + 1) / 2));
@@ -33,7 +34,7 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
     p.e = e;
     p.a = a;
     p.B = B;
-    p.D = D;
+    p.D = (int32_t)D;
     p.topo_index = topo_index;
     p.M = M;
     p.out_peak = out_peak;
@@ -42,17 +43,41 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
     p.out_seqs = out_seqs;
     p.out_lens = out_lens;
     p.words = (uint32_t)((D + 32) / 32);
-    const size_t smem = moc::interval_smem_bytes(p.words, K, topo_index == nullptr);
+    const bool plain = topo_index == nullptr;
+    const bool wide = g->sum_m > (int64_t)INT32_MAX / g->C;     // C * sum(m) bounds every partial usage sum
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
-    if (smem > cap)
+    const size_t base_b = moc::interval_clear_bytes(p.words, K, plain, wide ? 8 : 4), stage_b = moc::interval_stage_bytes(K);
+    if (base_b > cap || K > (int64_t)INT32_MAX / 2)
         return fail(MOC_ERR_ARG, "moc_check_intervals: domain of %lld events with %lld intervals needs %zu bytes of "
-                    "shared memory per block, the device offers %zu", (long long)D, (long long)K, smem, cap);
-    MOC_CUDA(cudaFuncSetAttribute(moc::check_intervals_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap));
+                    "shared memory per solution, the device offers %zu", (long long)D, (long long)K, base_b, cap);
+    // keep the solution on chip after the first pass while at least eight solutions per SM still fit
+    const bool stage = (base_b + stage_b) * 8 <= cap;
+    const size_t warp_b = base_b + (stage ? stage_b : 0);
+    p.warp_bytes = (uint32_t)warp_b;
+    // warps per block: the count that puts most warps on an SM (each block loses 1 KB to the system)
+    int wpb = 1, best = 0;
+    for (int k = 1; k <= moc::kIvMaxWarps; ++k) {
+        const size_t blk = warp_b * k + 1024;
+        const int fit = blk <= cap + 1024 ? (int)((g->smem_optin) / blk) * k : 0;
+        if (fit > best) { best = fit; wpb = k; }
+    }
+    const size_t smem = warp_b * wpb;
+    using Fn = void (*)(const moc::IntervalParams);
+    const int cp = g->C <= 2 ? 2 : (g->C <= 4 ? 4 : 8);
+    Fn table[2][3][2][2] = {
+#define MOC_IV_ROW(PL, CPV) {{(Fn)moc::check_intervals_kernel<PL, CPV, int32_t, false>, (Fn)moc::check_intervals_kernel<PL, CPV, int32_t, true>}, \
+                            {(Fn)moc::check_intervals_kernel<PL, CPV, int64_t, false>, (Fn)moc::check_intervals_kernel<PL, CPV, int64_t, true>}}
+        {MOC_IV_ROW(false, 2), MOC_IV_ROW(false, 4), MOC_IV_ROW(false, 8)},
+        {MOC_IV_ROW(true, 2), MOC_IV_ROW(true, 4), MOC_IV_ROW(true, 8)}
+#undef MOC_IV_ROW
+    };
+    Fn fn = table[plain ? 1 : 0][cp == 2 ? 0 : (cp == 4 ? 1 : 2)][wide ? 1 : 0][stage ? 1 : 0];
+    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap));
     int nb = 0;
-    MOC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, moc::check_intervals_kernel, moc::kIvThreads, smem));
+    MOC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, 32 * wpb, smem));
     if (nb < 1) return fail(MOC_ERR_CUDA, "moc_check_intervals: kernel does not fit on an SM");
-    const int grid = (int)std::min<int64_t>((int64_t)g->sm_count * nb, B);
-    moc::check_intervals_kernel<<<grid, moc::kIvThreads, smem, (cudaStream_t)stream>>>(p);
+    const int grid = (int)std::min<int64_t>((int64_t)g->sm_count * nb, ((int64_t)B + wpb - 1) / wpb);
+    fn<<<grid, 32 * wpb, smem, (cudaStream_t)stream>>>(p);
     MOC_CUDA(cudaGetLastError());
     launch_counter() = 1;
     return MOC_OK;
