@@ -53,7 +53,7 @@ __host__ __device__ inline size_t interval_bitmap_bytes(uint32_t words, bool pla
 __host__ __device__ inline size_t interval_clear_bytes(uint32_t words, int64_t K, bool plain, size_t mem_sz) {
     return interval_bitmap_bytes(words, plain) + (((size_t)(K + 2) * mem_sz + 15) & ~size_t(15));
 }
-__host__ __device__ inline size_t interval_stage_bytes(int64_t K) { return ((size_t)K * 8 + 15) & ~size_t(15); }
+__host__ __device__ inline size_t interval_stage_bytes(int64_t K, size_t pos_sz) { return ((size_t)K * 2 * pos_sz + 15) & ~size_t(15); }
 
 // exact test "x = j(j-1)/2 for an integer j >= jmin"; x >= 0
 __device__ __forceinline__ bool is_triangular_from(int64_t x, int64_t jmin) {
@@ -71,8 +71,9 @@ __device__ __forceinline__ void iv_add(int64_t* p, int64_t v) {
 
 // kPlain: plain model (Eq. 6) or staged model; CP: slots per node held in registers (>= C); MemT: type
 // of the usage sums (int32 when C * sum(m) < 2^31); kStage: the solution is kept in shared memory
-// after the first pass (otherwise the second pass reads it again through L1/L2).
-template <bool kPlain, int CP, typename MemT, bool kStage>
+// after the first pass (otherwise the second pass reads it again through L1/L2), as PosT (uint16 when
+// D < 65536).
+template <bool kPlain, int CP, typename MemT, bool kStage, typename PosT>
 __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const IntervalParams p) {
     extern __shared__ __align__(16) char smem[];
     const int lane = threadIdx.x & 31;
@@ -84,8 +85,8 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
     uint32_t* bm_all = bm_act + p.words;                               // plain model only
     uint32_t* rbase = bm_act + p.words * (kPlain ? 2u : 1u);
     MemT* delta = reinterpret_cast<MemT*>(ws + interval_bitmap_bytes(p.words, kPlain));
-    int32_t* sS = reinterpret_cast<int32_t*>(ws + interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)));
-    int32_t* sE = sS + K;
+    PosT* sS = reinterpret_cast<PosT*>(ws + interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)));
+    PosT* sE = sS + K;
     constexpr uint32_t kFull = 0xFFFFFFFFu;
     const int nz = (int)(interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)) >> 4);
 
@@ -102,7 +103,7 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         // ---- pass 1, per node: read the C slots; Eq. 8; Eqs. 1, 2, 3, 7; mark the starts in the bitmaps
         // (Eq. 6 / staged rule).  A start outside the domain marks nothing; the marks are used only when
         // Eq. 8 holds everywhere.
-        int32_t mask = 0, n_act = 0;
+        int32_t mask = 0, n_act = 0, n_distinct = 0;
         int64_t dur = 0;
         for (int32_t v = lane; v < n; v += 32) {
             int32_t sv[CP], ev[CP], av[CP];
@@ -130,8 +131,8 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                     const bool act = av[i] == 1;
                     if (act) { dur += wv; ++n_act; }
                     if (kStage) {
-                        sS[v * C + i] = act ? sv[i] : 0;
-                        sE[v * C + i] = ev[i];
+                        sS[v * C + i] = (PosT)(act ? sv[i] : 0);
+                        sE[v * C + i] = (PosT)ev[i];
                     }
                     if (in_dom) {
                         const uint32_t bit = 1u << (sv[i] & 31);
@@ -140,11 +141,15 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                             if (!kPlain && !((int64_t)sv[i] >= k && is_triangular_from((int64_t)sv[i] - k, k))) mask |= kIvStage;
                         }
                         if (kPlain) {
-                            // each node marks each of its distinct starts once: a bit found set belongs to another node
+                            // each node marks its distinct starts; Eq. 6 holds iff no two nodes marked the same
+                            // bit, i.e. iff the bitmap ends up with as many bits as marks were made
                             bool seen = false;
 #pragma unroll
                             for (int i2 = 0; i2 < i; ++i2) seen |= sv[i2] == sv[i];
-                            if (!seen && (atomicOr(&bm_all[sv[i] >> 5], bit) & bit)) mask |= kIvEq6;
+                            if (!seen) {
+                                atomicOr(&bm_all[sv[i] >> 5], bit);
+                                ++n_distinct;
+                            }
                         }
                     }
                 }
@@ -183,6 +188,12 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         }
         int32_t total_act = n_act;
         for (int d = 16; d > 0; d >>= 1) total_act += __shfl_xor_sync(kFull, total_act, d);
+        if (kPlain) {
+            int32_t bits = 0;
+            for (uint32_t i = lane; i < p.words; i += 32) bits += __popc(bm_all[i]);
+            bits = __reduce_add_sync(kFull, bits);
+            if (bits != __reduce_add_sync(kFull, n_distinct)) mask |= kIvEq6;
+        }
         const bool has_seq = R == total_act;
         int32_t* row = (p.out_seqs != nullptr && has_seq) ? p.out_seqs + (int64_t)b * K : nullptr;
         __syncwarp();
@@ -193,8 +204,8 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         // start (0 = inactive) and end of slot i of node v
         auto slot = [&](int32_t v, int32_t i, int32_t& s_out, int32_t& e_out) {
             if (kStage) {
-                s_out = sS[v * C + i];
-                e_out = sE[v * C + i];
+                s_out = (int32_t)sS[v * C + i];
+                e_out = (int32_t)sE[v * C + i];
             } else {
                 s_out = __ldg(ga + v * C + i) == 1 ? __ldg(gs + v * C + i) : 0;
                 e_out = __ldg(ge + v * C + i);

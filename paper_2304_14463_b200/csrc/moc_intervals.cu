@@ -46,7 +46,7 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
     const bool plain = topo_index == nullptr;
     const bool wide = g->sum_m > (int64_t)INT32_MAX / g->C;     // C * sum(m) bounds every partial usage sum
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
-    const size_t base_b = moc::interval_clear_bytes(p.words, K, plain, wide ? 8 : 4), stage_b = moc::interval_stage_bytes(K);
+    const size_t base_b = moc::interval_clear_bytes(p.words, K, plain, wide ? 8 : 4), stage_b = moc::interval_stage_bytes(K, D < 65536 ? 2 : 4);
     if (base_b > cap || K > (int64_t)INT32_MAX / 2)
         return fail(MOC_ERR_ARG, "moc_check_intervals: domain of %lld events with %lld intervals needs %zu bytes of "
                     "shared memory per solution, the device offers %zu", (long long)D, (long long)K, base_b, cap);
@@ -64,14 +64,17 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
     const size_t smem = warp_b * wpb;
     using Fn = void (*)(const moc::IntervalParams);
     const int cp = g->C <= 2 ? 2 : (g->C <= 4 ? 4 : 8);
-    Fn table[2][3][2][2] = {
-#define MOC_IV_ROW(PL, CPV) {{(Fn)moc::check_intervals_kernel<PL, CPV, int32_t, false>, (Fn)moc::check_intervals_kernel<PL, CPV, int32_t, true>}, \
-                            {(Fn)moc::check_intervals_kernel<PL, CPV, int64_t, false>, (Fn)moc::check_intervals_kernel<PL, CPV, int64_t, true>}}
+    const bool narrow = D < 65536;
+    Fn table[2][3][2][3] = {
+#define MOC_IV_ROW(PL, CPV) {{(Fn)moc::check_intervals_kernel<PL, CPV, int32_t, false, int32_t>, (Fn)moc::check_intervals_kernel<PL, CPV, int32_t, true, int32_t>, \
+                             (Fn)moc::check_intervals_kernel<PL, CPV, int32_t, true, uint16_t>},                                                            \
+                            {(Fn)moc::check_intervals_kernel<PL, CPV, int64_t, false, int32_t>, (Fn)moc::check_intervals_kernel<PL, CPV, int64_t, true, int32_t>, \
+                             (Fn)moc::check_intervals_kernel<PL, CPV, int64_t, true, uint16_t>}}
         {MOC_IV_ROW(false, 2), MOC_IV_ROW(false, 4), MOC_IV_ROW(false, 8)},
         {MOC_IV_ROW(true, 2), MOC_IV_ROW(true, 4), MOC_IV_ROW(true, 8)}
 #undef MOC_IV_ROW
     };
-    Fn fn = table[plain ? 1 : 0][cp == 2 ? 0 : (cp == 4 ? 1 : 2)][wide ? 1 : 0][stage ? 1 : 0];
+    Fn fn = table[plain ? 1 : 0][cp == 2 ? 0 : (cp == 4 ? 1 : 2)][wide ? 1 : 0][stage ? (narrow ? 2 : 1) : 0];
     MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap));
     int nb = 0;
     MOC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, 32 * wpb, smem));
