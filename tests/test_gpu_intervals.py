@@ -143,3 +143,31 @@ def test_interval_argument_errors(B):
         G.check_intervals(z, z, z, 1, D=7, topo_index=dev(np.arange(1, wl.n + 1)))   # staged needs D = n(n+1)/2
     with pytest.raises(B.MocError):
         G.check_intervals(z, z, z, 1, D=0)
+
+
+def test_interval_full_size_sampled(B):
+    """The benchmark's shape (headline graph, 16384 solutions, plain domain): every 37th solution is
+    compared with the oracle; the rest must agree with the copy of the same solution among them."""
+    nB, distinct = 16384, 128
+    wl = W.make(2, seed=1, B=distinct)
+    rng = np.random.default_rng(9)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    s, e, a, D, _ = build_batch(O, wl, rng, distinct, staged=False)
+    perm = rng.permutation(nB) % distinct
+    M = O.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    r = G.check_intervals(dev(s[perm]), dev(e[perm]), dev(a[perm]), M, D=D)
+    torch.cuda.synchronize()
+    mask, peak, dur, lens = (r[k].cpu().numpy() for k in ("mask", "peak", "dur", "lens"))
+    ref = {}
+    for b in range(0, nB, 37):
+        k = int(perm[b])
+        if k not in ref:
+            x = O.check_intervals(s[k], e[k], a[k], M, D=D)
+            ref[k] = (x["mask"], x["peak"], x["dur"])
+        assert (int(mask[b]), int(peak[b]), int(dur[b])) == ref[k], b
+    first = {}
+    for b in range(nB):
+        k = int(perm[b])
+        got = (int(mask[b]), int(peak[b]), int(dur[b]), int(lens[b]))
+        assert first.setdefault(k, got) == got, b

@@ -152,3 +152,16 @@ def test_search_restricted_kinds(B, kinds):
         S.set_kinds(0)
     with pytest.raises(B.MocError):
         S.set_kinds(8)
+
+
+def test_search_full_size(B):
+    """The benchmark's shape: the headline graph with 16384 chains, every chain compared."""
+    wl = W.make(2, seed=1)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G, O, S, OS = make_pair(B, wl, wl.seqs, wl.lens, M, seed=1)
+    assert OS.P == 16384
+    for g in (1, 3):
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"full size after {OS.generation}")
