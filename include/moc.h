@@ -209,6 +209,61 @@ int moc_check_intervals(const moc_graph* g, const int32_t* s, const int32_t* e, 
                         void* stream);
 
 /*
+ * ---- Incremental evaluation of edited sequences ------------------------------------------------
+ *
+ * A search looks at many sequences that differ from an evaluated one ("parent") by a single edit.
+ * Retention intervals are local to the copies of a node (Section 2: Eq. 3 orders the intervals of one
+ * node, Eq. 5 ties the end of an interval to the consumers of that node), so an edit of a copy of node
+ * x changes only the intervals of x and of the predecessors of x; the memory profile of Eq. 4 changes
+ * inside a window around them and is shifted elsewhere.  moc_cache_build evaluates the parents once and
+ * keeps their profile, its prefix and suffix maxima, the free steps and the positions of every node's
+ * copies on the device; moc_eval_edits then scores any number of edits of those parents from the
+ * cache.  The results are exactly those moc_eval_batch gives for the edited sequences.
+ *
+ * Limits: handles with C <= 2 (the setting of Section 4.3) and C*n <= 65534; per-node caps are honoured.
+ * The cache refers to the graph handle (which must outlive it, with unchanged C and caps) and owns
+ * about 12 + 12*sizeof(sum type) bytes per step and parent of device memory, allocated by
+ * moc_cache_create only.
+ */
+typedef struct moc_cache moc_cache; /* opaque */
+
+/* Room for up to max_parents parents.  Errors: MOC_ERR_ARG (C > 2, sequences too long for the
+ * on-chip state), MOC_ERR_CUDA, MOC_ERR_NOMEM. */
+int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out);
+
+/*
+ * Evaluates P parents (seqs, lens: DEVICE, packed as for moc_eval_batch) against budget M and fills
+ * the cache; parent k of later moc_eval_edits calls is sequence k of this call.  out_peak, out_dur,
+ * out_status (DEVICE, P each, any may be NULL) receive the same values as moc_eval_batch.
+ * Asynchronous on `stream`; two kernels; no allocation.  1 <= P <= max_parents.
+ */
+int moc_cache_build(moc_cache* c, const int32_t* seqs, const int32_t* lens, int32_t P, int64_t M,
+                    int64_t* out_peak, int64_t* out_dur, int32_t* out_status, void* stream);
+
+/*
+ * Scores B edits.  Edit b takes parent parent[b] (sequence of T steps) and
+ *     op[b] = 0  inserts a further copy of node seq[q[b]] in front of index j[b], 0 <= j <= T;
+ *     op[b] = 1  removes step q[b]  (j[b] is ignored);
+ *     op[b] = 2  removes step q[b] and puts its node back in front of index j[b] of the shortened
+ *                sequence, 0 <= j <= T-1;
+ * with 0 <= q[b] < T: the edits of the search entry points.  All arrays DEVICE, B entries.
+ *   out_peak, out_dur, out_status: what moc_eval_batch reports for the edited sequence (status
+ *   1 / 0 / -1 / -2 with the same sentinels).  Two more cases: an edit whose parent index, op, q or
+ *   j is out of range gets status -2 (peak = dur = -1); an edit of a parent whose own status is
+ *   negative gets status MOC_STATUS_PARENT_INVALID (-3, peak = dur = -1): such a parent has no
+ *   profile to start from, evaluate the edited sequence with moc_eval_batch.
+ * Asynchronous on `stream` (ordered after moc_cache_build on the same stream); one kernel; no
+ * allocation.
+ */
+#define MOC_STATUS_PARENT_INVALID (-3)
+int moc_eval_edits(const moc_cache* c, const int32_t* parent, const int32_t* op, const int32_t* q,
+                   const int32_t* j, int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur,
+                   int32_t* out_status, void* stream);
+
+/* Frees the cache; NULL is accepted.  Synchronise its streams first. */
+void moc_cache_destroy(moc_cache* c);
+
+/*
  * ---- Local search over sequences (Section 3, "Optimization in Two Phases") -------------------------
  *
  * P independent chains each hold one sequence and its evaluation.  One generation proposes, for

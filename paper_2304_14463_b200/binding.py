@@ -20,7 +20,8 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_eval_batch", "moc_eval_batch_host", "moc_mem_profile", "moc_graph_set_launch",
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
-           "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals"]
+           "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals",
+           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -52,6 +53,14 @@ lib.moc_graph_set_timing_events.restype = ctypes.c_int
 lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
 lib.moc_check_intervals.restype = ctypes.c_int
 lib.moc_check_intervals.argtypes = [_P, _P, _P, _P, _i32, _i64, _P, _i64, _P, _P, _P, _P, _P, _P]
+lib.moc_cache_create.restype = ctypes.c_int
+lib.moc_cache_create.argtypes = [_P, _i32, ctypes.POINTER(_P)]
+lib.moc_cache_build.restype = ctypes.c_int
+lib.moc_cache_build.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_eval_edits.restype = ctypes.c_int
+lib.moc_eval_edits.argtypes = [_P, _P, _P, _P, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_cache_destroy.restype = None
+lib.moc_cache_destroy.argtypes = [_P]
 lib.moc_search_create.restype = ctypes.c_int
 lib.moc_search_create.argtypes = [_P, _P, _P, _i32, _i64, ctypes.c_uint64, ctypes.c_uint32, _P, ctypes.POINTER(_P)]
 lib.moc_search_run.restype = ctypes.c_int
@@ -417,3 +426,50 @@ class Search:
         b = b.cpu().numpy()
         return dict(index=int(b[0]), seq=seq[:int(b[1])].cpu().numpy(), peak=int(b[2]), dur=int(b[3]),
                     status=int(b[4]), accepted=int(b[5]))
+
+
+MOC_STATUS_PARENT_INVALID = -3
+
+
+class EditCache:
+    """Owns a moc_cache handle: evaluated parents on the device, from which single edits are scored."""
+
+    def __init__(self, graph: Graph, max_parents):
+        self.graph = graph
+        h = _P()
+        _check(lib.moc_cache_create(graph.h, int(max_parents), ctypes.byref(h)), "moc_cache_create")
+        self.h = h
+
+    def close(self, _destroy=lib.moc_cache_destroy):
+        if getattr(self, "h", None):
+            _destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def build(self, seqs, lens, M):
+        """Device tensors (packed parents) -> (peak, dur, status) device tensors of the parents."""
+        import torch
+        P = lens.numel()
+        peak = torch.empty(P, dtype=torch.int64, device=lens.device)
+        dur = torch.empty(P, dtype=torch.int64, device=lens.device)
+        st = torch.empty(P, dtype=torch.int32, device=lens.device)
+        rc = lib.moc_cache_build(self.h, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"), P, int(M),
+                                 _dev(peak, torch.int64, "peak"), _dev(dur, torch.int64, "dur"),
+                                 _dev(st, torch.int32, "status"), _stream())
+        _check(rc, "moc_cache_build")
+        return peak, dur, st
+
+    def eval_edits(self, parent, op, q, j, M, out=None):
+        """int32 device tensors of B edits -> (peak, dur, status) device tensors."""
+        import torch
+        B = parent.numel()
+        if out is None:
+            out = (torch.empty(B, dtype=torch.int64, device=parent.device), torch.empty(B, dtype=torch.int64, device=parent.device),
+                   torch.empty(B, dtype=torch.int32, device=parent.device))
+        rc = lib.moc_eval_edits(self.h, _dev(parent, torch.int32, "parent"), _dev(op, torch.int32, "op"),
+                                _dev(q, torch.int32, "q"), _dev(j, torch.int32, "j"), B, int(M),
+                                _dev(out[0], torch.int64, "peak"), _dev(out[1], torch.int64, "dur"),
+                                _dev(out[2], torch.int32, "status"), _stream())
+        _check(rc, "moc_eval_edits")
+        return out

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoc_b200.so")
-SOURCES = ["moc_api.cu", "moc_search.cu", "moc_intervals.cu"]
-HEADERS = ["moc_kernels.cuh", "moc_pair_kernel.cuh", "moc_host.cuh", "moc_search_kernels.cuh", "moc_interval_kernels.cuh", os.path.join("..", "..", "include", "moc.h")]
+SOURCES = ["moc_api.cu", "moc_search.cu", "moc_intervals.cu", "moc_edits.cu"]
+HEADERS = ["moc_kernels.cuh", "moc_pair_kernel.cuh", "moc_host.cuh", "moc_search_kernels.cuh", "moc_interval_kernels.cuh", "moc_edit_kernels.cuh", os.path.join("..", "..", "include", "moc.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "--use_fast_math"]
 
@@ -28,7 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".{os.getpid()}.tmp"
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-          ["-t", "3", "-o", tmp] + [os.path.join(CSRC, f) for f in SOURCES]
+          ["-t", "4", "-o", tmp] + [os.path.join(CSRC, f) for f in SOURCES]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
     return LIB

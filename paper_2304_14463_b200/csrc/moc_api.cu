@@ -427,6 +427,25 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     };
     up((void**)&g->d_succ_start, succ_start.data(), ((size_t)n + 1) * 4);
     up((void**)&g->d_succ, succ.data(), (size_t)ne * 4);
+    {
+        // predecessor lists (grouped by consumer) and the total output size of the sinks
+        std::vector<int32_t> pred_start, pred;
+        try {
+            pred_start.assign((size_t)n + 1, 0);
+            pred.resize((size_t)std::max<int64_t>(ne, 1));
+            for (int64_t k = 0; k < ne; ++k) pred_start[(keys[k] & 0xFFFFFFFFu) + 1]++;
+            for (int32_t v = 0; v < n; ++v) pred_start[v + 1] += pred_start[v];
+            std::vector<int32_t> fill(pred_start.begin(), pred_start.end() - 1);
+            for (int64_t k = 0; k < ne; ++k) pred[fill[keys[k] & 0xFFFFFFFFu]++] = (int32_t)(keys[k] >> 32);
+        } catch (const std::bad_alloc&) {
+            moc_graph_destroy(g);
+            return fail(MOC_ERR_NOMEM, "host allocation failed");
+        }
+        for (int32_t v = 0; v < n; ++v)
+            if (succ_start[v + 1] == succ_start[v]) g->sink_m += m[v];
+        up((void**)&g->d_pred_start, pred_start.data(), ((size_t)n + 1) * 4);
+        up((void**)&g->d_pred, pred.data(), (size_t)ne * 4);
+    }
     up((void**)&g->d_w, w, (size_t)n * 8);
     up((void**)&g->d_m64, m, (size_t)n * 8);
     up((void**)&g->d_m32, m32.data(), (size_t)n * 4);
@@ -618,6 +637,8 @@ void moc_graph_destroy(moc_graph* g) {
     DeviceGuard dg(g->device);
     cudaFree(g->d_succ_start);
     cudaFree(g->d_succ);
+    cudaFree(g->d_pred_start);
+    cudaFree(g->d_pred);
     cudaFree(g->d_w);
     cudaFree(g->d_m64);
     cudaFree(g->d_m32);

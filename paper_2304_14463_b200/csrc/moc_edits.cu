@@ -1,0 +1,180 @@
+// Host side of the incremental evaluation (moc_cache_*, moc_eval_edits; declared in include/moc.h):
+// the cache of evaluated parents on the device and the two launches.
+#include <algorithm>
+#include <new>
+
+#include "moc_host.cuh"
+#include "moc_edit_kernels.cuh"
+
+using namespace moc_host;
+
+struct moc_cache {
+    const moc_graph* g = nullptr;
+    int device = 0;
+    int32_t max_parents = 0;
+    bool wide = false;
+    char* d_block = nullptr;
+    int64_t* d_offs = nullptr;     // max_parents + 1
+    moc::EditCacheDev c{};
+    size_t warp_bytes = 0;
+    int wpb = 0, grid_cap = 0;
+};
+
+namespace {
+size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
+}  // namespace
+
+extern "C" {
+
+int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
+    clear_error();
+    if (out) *out = nullptr;
+    if (!g || !out || max_parents < 1) return fail(MOC_ERR_ARG, "moc_cache_create: null pointer or max_parents < 1");
+    if (g->C > 2) return fail(MOC_ERR_ARG, "moc_cache_create: the incremental evaluation covers C <= 2 (handle has C = %d)", g->C);
+    const int64_t max_T = (int64_t)g->C * g->n;
+    if (max_T > 65534) return fail(MOC_ERR_ARG, "moc_cache_create: sequences of up to %lld steps exceed 65534", (long long)max_T);
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    moc_cache* h = new (std::nothrow) moc_cache();
+    if (!h) return fail(MOC_ERR_NOMEM, "host allocation failed");
+    h->g = g;
+    h->device = g->device;
+    h->max_parents = max_parents;
+    h->wide = g->sum_m > (int64_t)INT32_MAX / g->C;
+    const size_t msz = h->wide ? 8 : 4;
+    const int32_t stride = (int32_t)((max_T + 3) & ~int64_t(3)), occ_stride = (g->n + 1 + 3) & ~3;
+    h->warp_bytes = moc::edit_warp_bytes(occ_stride, stride, msz);
+    const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
+    if (h->warp_bytes > cap) {
+        delete h;
+        return fail(MOC_ERR_ARG, "moc_cache_create: %zu bytes of shared memory per sequence exceed the device's %zu", h->warp_bytes, cap);
+    }
+    // warps per block: the count that puts most warps on an SM
+    int best = 0;
+    for (int k = 1; k <= moc::kEditThreads / 32; ++k) {
+        const size_t blk = h->warp_bytes * k + 1024;
+        const int fit = blk <= cap + 1024 ? (int)(g->smem_optin / blk) * k : 0;
+        if (fit > best) { best = fit; h->wpb = k; }
+    }
+    h->grid_cap = g->sm_count * std::max(1, best / h->wpb);
+    const size_t P = (size_t)max_parents, S = (size_t)stride;
+    const size_t o_row = 0, o_fre = o_row + up256(P * S * 4), o_prof = o_fre + up256(P * S * 4), o_pm = o_prof + up256(P * S * msz),
+                 o_sm = o_pm + up256(P * S * msz), o_occ = o_sm + up256(P * S * msz), o_len = o_occ + up256(P * occ_stride * 4),
+                 o_st = o_len + up256(P * 4), o_peak = o_st + up256(P * 4), o_dur = o_peak + up256(P * 8),
+                 o_offs = o_dur + up256(P * 8), total = o_offs + up256((P + 1) * 8);
+    cudaError_t e = cudaMalloc((void**)&h->d_block, total);
+    if (e != cudaSuccess) {
+        delete h;
+        cudaGetLastError();
+        return fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, "moc_cache_create: %s", cudaGetErrorString(e));
+    }
+    char* b = h->d_block;
+    moc::EditCacheDev& c = h->c;
+    c.n = g->n;
+    c.C = g->C;
+    c.P = 0;
+    c.stride = stride;
+    c.occ_stride = occ_stride;
+    c.max_T = (int32_t)max_T;
+    c.succ_start = g->d_succ_start;
+    c.succ = g->d_succ;
+    c.pred_start = g->d_pred_start;
+    c.pred = g->d_pred;
+    c.w = g->d_w;
+    c.m = g->d_m64;
+    c.cap = g->d_cap;
+    c.sink_m = g->sink_m;
+    c.row = (int32_t*)(b + o_row);
+    c.fre = (int32_t*)(b + o_fre);
+    c.prof = b + o_prof;
+    c.pm = b + o_pm;
+    c.sm = b + o_sm;
+    c.occ = (uint32_t*)(b + o_occ);
+    c.len = (int32_t*)(b + o_len);
+    c.status = (int32_t*)(b + o_st);
+    c.peak = (int64_t*)(b + o_peak);
+    c.dur = (int64_t*)(b + o_dur);
+    h->d_offs = (int64_t*)(b + o_offs);
+    *out = h;
+    return MOC_OK;
+}
+
+int moc_cache_build(moc_cache* h, const int32_t* seqs, const int32_t* lens, int32_t P, int64_t M, int64_t* out_peak,
+                    int64_t* out_dur, int32_t* out_status, void* stream) {
+    clear_error();
+    launch_counter() = 0;
+    if (!h || !seqs || !lens || P < 1 || P > h->max_parents)
+        return fail(MOC_ERR_ARG, "moc_cache_build: null pointer, or P outside [1, max_parents = %d]", h ? h->max_parents : 0);
+    if (h->g->C != h->c.C) return fail(MOC_ERR_ARG, "moc_cache_build: the graph's C changed after the cache was created");
+    DeviceGuard dg(h->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", h->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    h->c.P = P;
+    h->c.cap = h->g->d_cap;
+    moc::PrepParams p{};
+    p.c = h->c;
+    p.seqs = seqs;
+    p.lens = lens;
+    p.offs = h->d_offs;
+    p.M = M;
+    p.out_peak = out_peak;
+    p.out_dur = out_dur;
+    p.out_status = out_status;
+    p.warp_bytes = (uint32_t)h->warp_bytes;
+    moc::offsets_kernel<<<(P + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, P, h->d_offs);
+    auto fn = h->wide ? moc::edit_prepare_kernel<int64_t> : moc::edit_prepare_kernel<int32_t>;
+    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
+    const int grid = (int)std::min<int64_t>(h->grid_cap, ((int64_t)P + h->wpb - 1) / h->wpb);
+    fn<<<grid, 32 * h->wpb, h->warp_bytes * h->wpb, st>>>(p);
+    MOC_CUDA(cudaGetLastError());
+    launch_counter() = 2;
+    return MOC_OK;
+}
+
+int moc_eval_edits(const moc_cache* h, const int32_t* parent, const int32_t* op, const int32_t* q, const int32_t* j,
+                   int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_status, void* stream) {
+    clear_error();
+    launch_counter() = 0;
+    if (!h || B < 0) return fail(MOC_ERR_ARG, "moc_eval_edits: null handle or B < 0");
+    if (B == 0) return MOC_OK;
+    if (!parent || !op || !q || !j || !out_peak || !out_dur || !out_status) return fail(MOC_ERR_ARG, "moc_eval_edits: null array");
+    if (h->c.P < 1) return fail(MOC_ERR_ARG, "moc_eval_edits: the cache holds no parents (call moc_cache_build first)");
+    DeviceGuard dg(h->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", h->device);
+    moc::EditParams p{};
+    p.c = h->c;
+    p.parent = parent;
+    p.op = op;
+    p.q = q;
+    p.j = j;
+    p.B = B;
+    p.M = M;
+    p.out_peak = out_peak;
+    p.out_dur = out_dur;
+    p.out_status = out_status;
+    const size_t msz = h->wide ? 8 : 4;
+    const size_t warp_b = 2 * ((((size_t)h->c.stride + 4) * msz + 15) & ~size_t(15));
+    p.warp_bytes = (uint32_t)warp_b;
+    const int wpb = moc::kEditThreads / 32;
+    const size_t smem = warp_b * wpb;
+    auto fn = h->wide ? moc::edit_eval_kernel<int64_t> : moc::edit_eval_kernel<int32_t>;
+    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
+    if (smem > h->g->smem_optin - 1024) return fail(MOC_ERR_ARG, "moc_eval_edits: sequences too long for this build");
+    int nb = 0;
+    MOC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, moc::kEditThreads, smem));
+    if (nb < 1) return fail(MOC_ERR_CUDA, "moc_eval_edits: kernel does not fit on an SM");
+    const int grid = (int)std::min<int64_t>((int64_t)h->g->sm_count * nb, ((int64_t)B + wpb - 1) / wpb);
+    fn<<<grid, moc::kEditThreads, smem, (cudaStream_t)stream>>>(p);
+    MOC_CUDA(cudaGetLastError());
+    launch_counter() = 1;
+    return MOC_OK;
+}
+
+void moc_cache_destroy(moc_cache* h) {
+    if (!h) return;
+    DeviceGuard dg(h->device);
+    cudaFree(h->d_block);
+    delete h;
+}
+
+}  // extern "C"

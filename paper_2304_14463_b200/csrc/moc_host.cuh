@@ -70,6 +70,9 @@ struct moc_graph {
     int64_t sum_m = 0, sum_w = 0;
     int32_t* d_succ_start = nullptr;
     int32_t* d_succ = nullptr;
+    int32_t* d_pred_start = nullptr;     // predecessor lists (CSR), for the incremental evaluation
+    int32_t* d_pred = nullptr;
+    int64_t sink_m = 0;                   // sum of m over the nodes without successors
     int64_t* d_w = nullptr;
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;

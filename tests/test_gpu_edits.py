@@ -1,0 +1,151 @@
+"""Parity of the incremental evaluation (moc_cache_build + moc_eval_edits, through the C ABI) with the
+oracle: every edited sequence is built on the CPU (the oracle's edit, pinned in test_search_oracle.py)
+and evaluated from scratch by the oracle's evaluator; peak, duration and status must be identical."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OracleGraph
+from paper_2304_14463_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+BIG = 1 << 60
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2304_14463_b200 import build
+    build.build()
+    from paper_2304_14463_b200 import binding
+    return binding
+
+
+def dev(a, dtype=torch.int32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype).cuda()
+
+
+def reference(O, seqs, lens, parent, op, q, j, M, parent_status):
+    offs = np.concatenate([[0], np.cumsum(np.clip(lens, 0, None))])
+    out = np.zeros((len(parent), 3), np.int64)
+    for b in range(len(parent)):
+        c = parent[b]
+        if c < 0 or c >= len(lens):
+            out[b] = (-1, -1, -2)
+            continue
+        if parent_status[c] < 0:
+            out[b] = (-1, -1, -3)
+            continue
+        row = seqs[offs[c]:offs[c + 1]]
+        T = len(row)
+        ok = 0 <= op[b] <= 2 and 0 <= q[b] < T and (op[b] == 1 or 0 <= j[b] <= (T if op[b] == 0 else T - 1))
+        if not ok:
+            out[b] = (-1, -1, -2)
+            continue
+        child = oracle.mutate(row, int(op[b]), int(q[b]), int(j[b]))
+        r = O.eval(child, M)
+        out[b] = (r["peak"], r["dur"], r["status"])
+    return out
+
+
+def run_case(B, wl, seqs, lens, M, parent, op, q, j, caps=None, what=""):
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    if caps is not None:
+        O.set_caps(caps)
+        G.set_caps(caps)
+    cache = B.EditCache(G, len(lens))
+    pk, du, st = cache.build(dev(seqs), dev(lens), M)
+    torch.cuda.synchronize()
+    rp, rd, rs, _ = O.eval_batch(seqs, lens, M)
+    assert (pk.cpu().numpy() == rp).all() and (du.cpu().numpy() == rd).all() and (st.cpu().numpy() == rs).all(), what
+    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    torch.cuda.synchronize()
+    got = np.stack([got[0].cpu().numpy(), got[1].cpu().numpy(), got[2].cpu().numpy().astype(np.int64)], 1)
+    want = reference(O, seqs, lens, parent, op, q, j, M, rs)
+    bad = np.nonzero((got != want).any(1))[0]
+    assert len(bad) == 0, f"{what}: {len(bad)} of {len(parent)} edits differ; first: edit {bad[0]} parent {parent[bad[0]]} " \
+                          f"op {op[bad[0]]} q {q[bad[0]]} j {j[bad[0]]}: gpu {got[bad[0]]} oracle {want[bad[0]]}"
+    return want
+
+
+def random_edits(rng, lens, nE):
+    parent = rng.integers(0, len(lens), nE).astype(np.int32)
+    op = rng.integers(0, 3, nE).astype(np.int32)
+    T = lens[parent]
+    q = (rng.integers(0, 1 << 30, nE) % np.maximum(T, 1)).astype(np.int32)
+    j = (rng.integers(0, 1 << 30, nE) % np.where(op == 0, T + 1, np.maximum(T, 1))).astype(np.int32)
+    return parent, op, q, j
+
+
+def test_edits_tiny_exhaustive(B):
+    """Every edit of several sequences on small graphs (all q, all j, all three kinds)."""
+    rng = np.random.default_rng(0)
+    for n, edges in [(4, [(0, 1), (1, 2), (2, 3), (0, 3)]), (5, [(0, 1), (0, 2), (1, 3), (2, 3), (3, 4)]),
+                     (5, [(0, 2), (1, 2), (2, 3), (2, 4)]), (3, [])]:
+        class WL:
+            pass
+        wl = WL()
+        wl.n, wl.edges, wl.C = n, np.array(edges, np.int32).reshape(-1, 2), 2
+        wl.w = rng.integers(1, 9, n).astype(np.int64)
+        wl.m = rng.integers(1, 20, n).astype(np.int64)
+        rows = [list(range(n))]
+        for _ in range(6):                       # valid sequences with extra copies
+            r = list(range(n))
+            for v in range(n):
+                if rng.random() < 0.5:
+                    r.insert(int(rng.integers(r.index(v) + 1, len(r) + 1)), v)
+            rows.append(r)
+        rows.append(list(range(n))[::-1] if edges else list(range(n)))     # an invalid parent (when there are edges)
+        seqs = np.array([x for r in rows for x in r], np.int32)
+        lens = np.array([len(r) for r in rows], np.int32)
+        parent, op, q, j = [], [], [], []
+        for c, r in enumerate(rows):
+            for o in range(3):
+                for qq in range(len(r)):
+                    for jj in range(len(r) + 1 if o == 0 else (1 if o == 1 else len(r))):
+                        parent.append(c); op.append(o); q.append(qq); j.append(jj)
+        M = int(wl.m.sum()) * 2 // 3
+        run_case(B, wl, seqs, lens, M, np.array(parent, np.int32), np.array(op, np.int32), np.array(q, np.int32),
+                 np.array(j, np.int32), what=f"tiny n={n}")
+
+
+@pytest.mark.parametrize("idx,P,nE", [(0, 256, 20000), (1, 128, 20000), (2, 64, 12000)])
+def test_edits_random(B, idx, P, nE):
+    """Random edits of workload sequences (1/16 of the parents damaged), plus malformed edit records."""
+    wl = W.make(idx, seed=2, B=P)
+    rng = np.random.default_rng(10 + idx)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=6, frac=1 / 16)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    parent, op, q, j = random_edits(rng, np.clip(lens, 0, None), nE)
+    # malformed records
+    parent[:4] = [-1, P, 0, 0]
+    op[4:6] = [3, -1]
+    q[6] = lens[parent[6]]
+    j[7] = lens[parent[7]] + 5
+    want = run_case(B, wl, seqs, lens, M, parent, op, q, j, what=f"config {idx}")
+    seen = set(want[:, 2].tolist())
+    assert {1, -1, -2, -3} <= seen or {0, -1, -2, -3} <= seen
+
+
+def test_edits_node_caps_and_wide(B):
+    wl = W.make(1, seed=3, B=64)
+    rng = np.random.default_rng(5)
+    caps = np.where(rng.random(wl.n) < 0.5, 1, 2).astype(np.int32)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    # parents that respect the caps: the identity order and orders with copies of uncapped nodes only
+    rows = []
+    for _ in range(64):
+        r = list(range(wl.n))
+        for v in np.nonzero(caps == 2)[0]:
+            if rng.random() < 0.3:
+                r.insert(int(rng.integers(r.index(v) + 1, len(r) + 1)), int(v))
+        rows.append(r)
+    seqs = np.array([x for r in rows for x in r], np.int32)
+    lens = np.array([len(r) for r in rows], np.int32)
+    run_case(B, wl, seqs, lens, M, *random_edits(rng, lens, 8000), caps=caps, what="caps")
+    # 64-bit sums
+    wl.m = wl.m * (1 << 33)
+    run_case(B, wl, seqs, lens, M * (1 << 33), *random_edits(rng, lens, 4000), what="wide")
