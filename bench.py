@@ -328,6 +328,99 @@ def run_intervals(args):
     print(json.dumps(line))
 
 
+def run_edits(args):
+    """Throughput of the incremental evaluation: random single edits of the headline batch's sequences,
+    scored from the cached parents.  Prints a JSON line of its own."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --mode edits needs a CUDA device")
+    torch.cuda.set_device(0)
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2304_14463_b200 import binding, workloads
+    base = workloads.make(WORKLOAD_IDX, seed=1)
+    P, per_parent = base.B, 16
+    G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
+    M = binding.budget_from_peak(G.no_remat_peak(), PCT)
+    cache = binding.EditCache(G, P)
+    d_seqs, d_lens = torch.from_numpy(base.seqs).cuda(), torch.from_numpy(base.lens).cuda()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cache.build(d_seqs, d_lens, M)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    cache.build(d_seqs, d_lens, M)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    build_ms = e0.elapsed_time(e1)
+    nE = P * per_parent
+    ring = []
+    for k in range(4):
+        rng = np.random.default_rng(k)
+        parent = rng.permutation(nE).astype(np.int32) % P
+        T = base.lens[parent]
+        op = rng.integers(0, 3, nE).astype(np.int32)
+        q = (rng.integers(0, 1 << 30, nE) % T).astype(np.int32)
+        j = (rng.integers(0, 1 << 30, nE) % np.where(op == 0, T + 1, T)).astype(np.int32)
+        ring.append([torch.from_numpy(x).cuda() for x in (parent, op, q, j)] + [parent, op, q, j])
+    out = (torch.empty(nE, dtype=torch.int64, device="cuda"), torch.empty(nE, dtype=torch.int64, device="cuda"),
+           torch.empty(nE, dtype=torch.int32, device="cuda"))
+    window = torch.zeros(nE, dtype=torch.int32, device="cuda")
+    steps, warm = (100 if args.steps is None else args.steps), max(3, 5 if args.warmup is None else args.warmup)
+    for i in range(warm):
+        r = ring[i % 4]
+        cache.eval_edits(r[0], r[1], r[2], r[3], M, out=out, window=window)
+    torch.cuda.synchronize()
+    mean_window = float(window.double().mean())
+    with ClockSampler(0) as clocks:
+        e0.record(stream)
+        for i in range(steps):
+            r = ring[i % 4]
+            cache.eval_edits(r[0], r[1], r[2], r[3], M, out=out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    last = ring[(steps - 1) % 4]
+    st = out[2].cpu().numpy()
+    mean_T = float(base.lens.mean())
+    msz = 8 if G.info()["wide"] else 4
+    # per edit: the record (16 B), the result (20 B), the cached usage over the recomputed window, two
+    # extrema, and about a dozen position / free-step words of the edited node and its neighbours
+    alg_bytes = nE * (36 + msz * mean_window + 2 * msz + 64)
+    peak_gbs, peak_kind = load_peaks()
+    line = {"metric": "edits_scored_per_s_n442", "value": nE / (ms * 1e-3), "unit": "edits/s", "n_gpus": 1, "steps": steps,
+            "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64" if msz == 8 else "int32", "data": "synthetic",
+            "config": {"workload": f"moc_eval_edits on {base.name}: n={base.n} C={base.C}, {P} cached parents, {per_parent} random "
+                                   f"edits each (insert / delete / move), M={PCT}% of no-remat peak",
+                       "cold_l2": f"cache of the parents: {P * (12 + 3 * msz) * (2 * base.n) / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
+                       "mean_T": mean_T, "mean_recomputed_steps": mean_window},
+            "equivalent_schedule_steps_per_s": nE * mean_T / (ms * 1e-3), "cache_build_ms": build_ms, "gpu_launches": steps,
+            "status_counts": {str(k): int((st == k).sum()) for k in (1, 0, -1, -2, -3)},
+            "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
+                         "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "algorithmic_bytes_per_launch": alg_bytes},
+            "clocks": clocks.summary()}
+    if not args.no_cpu_baseline:
+        import oracle
+        from oracle import OracleGraph
+        O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
+        offs = np.concatenate([[0], np.cumsum(base.lens)])
+        pk, du = out[0].cpu().numpy(), out[1].cpu().numpy()
+        t0, k, same = time.perf_counter(), 0, True
+        while time.perf_counter() - t0 < 8.0 and k < nE:
+            c = last[4][k]
+            child = oracle.mutate(base.seqs[offs[c]:offs[c + 1]], int(last[5][k]), int(last[6][k]), int(last[7][k]))
+            r = O.eval(child, M)
+            same = same and (r["peak"], r["dur"], r["status"]) == (int(pk[k]), int(du[k]), int(st[k]))
+            k += 1
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": k / dt, "unit": "edits/s", "cores": 1, "kind": "oracle",
+                                "sample": f"the first {k} edits of the last batch: edit + full evaluation, one core"}
+        line["parity_sample"] = bool(same)
+    print(json.dumps(line))
+
+
 def time_oracle(base, M, budget_s=6.0):
     from oracle import OracleGraph
     O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
@@ -358,15 +451,17 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", type=int, default=WORKLOAD_IDX,
                     help="index 0..4 of the configuration to time (default: the headline one)")
-    ap.add_argument("--mode", default="eval", choices=["eval", "search", "intervals"],
+    ap.add_argument("--mode", default="eval", choices=["eval", "search", "intervals", "edits"],
                     help="eval: the headline evaluation metric; search: generations of the search entry points; "
-                         "intervals: the interval-form checker")
+                         "intervals: the interval-form checker; edits: the incremental evaluation of single edits")
     ap.add_argument("--chains", type=int, default=32768, help="--mode search: number of chains")
     args = ap.parse_args()
     if args.mode == "search" and args.impl != "reference":
         return run_search(args)
     if args.mode == "intervals" and args.impl != "reference":
         return run_intervals(args)
+    if args.mode == "edits" and args.impl != "reference":
+        return run_edits(args)
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

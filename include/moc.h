@@ -252,13 +252,15 @@ int moc_cache_build(moc_cache* c, const int32_t* seqs, const int32_t* lens, int3
  *   j is out of range gets status -2 (peak = dur = -1); an edit of a parent whose own status is
  *   negative gets status MOC_STATUS_PARENT_INVALID (-3, peak = dur = -1): such a parent has no
  *   profile to start from, evaluate the edited sequence with moc_eval_batch.
+ *   out_window (DEVICE, B int32, may be NULL): number of steps of the edited sequence whose usage had
+ *   to be recomputed (0 when the edit was refused before that point): the cost of the edit.
  * Asynchronous on `stream` (ordered after moc_cache_build on the same stream); one kernel; no
  * allocation.
  */
 #define MOC_STATUS_PARENT_INVALID (-3)
 int moc_eval_edits(const moc_cache* c, const int32_t* parent, const int32_t* op, const int32_t* q,
                    const int32_t* j, int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur,
-                   int32_t* out_status, void* stream);
+                   int32_t* out_status, int32_t* out_window, void* stream);
 
 /* Frees the cache; NULL is accepted.  Synchronise its streams first. */
 void moc_cache_destroy(moc_cache* c);

@@ -58,7 +58,7 @@ lib.moc_cache_create.argtypes = [_P, _i32, ctypes.POINTER(_P)]
 lib.moc_cache_build.restype = ctypes.c_int
 lib.moc_cache_build.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_eval_edits.restype = ctypes.c_int
-lib.moc_eval_edits.argtypes = [_P, _P, _P, _P, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_eval_edits.argtypes = [_P, _P, _P, _P, _P, _i32, _i64, _P, _P, _P, _P, _P]
 lib.moc_cache_destroy.restype = None
 lib.moc_cache_destroy.argtypes = [_P]
 lib.moc_search_create.restype = ctypes.c_int
@@ -460,8 +460,9 @@ class EditCache:
         _check(rc, "moc_cache_build")
         return peak, dur, st
 
-    def eval_edits(self, parent, op, q, j, M, out=None):
-        """int32 device tensors of B edits -> (peak, dur, status) device tensors."""
+    def eval_edits(self, parent, op, q, j, M, out=None, window=None):
+        """int32 device tensors of B edits -> (peak, dur, status) device tensors; window: optional int32
+        device tensor that receives the number of recomputed steps per edit."""
         import torch
         B = parent.numel()
         if out is None:
@@ -470,6 +471,7 @@ class EditCache:
         rc = lib.moc_eval_edits(self.h, _dev(parent, torch.int32, "parent"), _dev(op, torch.int32, "op"),
                                 _dev(q, torch.int32, "q"), _dev(j, torch.int32, "j"), B, int(M),
                                 _dev(out[0], torch.int64, "peak"), _dev(out[1], torch.int64, "dur"),
-                                _dev(out[2], torch.int32, "status"), _stream())
+                                _dev(out[2], torch.int32, "status"),
+                                _dev(window, torch.int32, "window") if window is not None else None, _stream())
         _check(rc, "moc_eval_edits")
         return out

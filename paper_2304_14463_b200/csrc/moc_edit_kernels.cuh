@@ -256,6 +256,7 @@ struct EditParams {
     int64_t* out_peak;
     int64_t* out_dur;
     int32_t* out_status;
+    int32_t* out_window;        // may be null: steps of the child whose usage was recomputed
     uint32_t warp_bytes;        // two arrays of stride + 4 MemT
 };
 
@@ -278,7 +279,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
 
     for (int32_t e = blockIdx.x * wpb + warp; e < p.B; e += gridDim.x * wpb) {
         int64_t out_pk = -1, out_du = -1;
-        int32_t out_st = -2;
+        int32_t out_st = -2, out_win = 0;
         const int32_t ci = __ldg(&p.parent[e]), o = __ldg(&p.op[e]), qq = __ldg(&p.q[e]), jj = __ldg(&p.j[e]);
         bool go = ci >= 0 && ci < c.P;
         int32_t T = 0;
@@ -418,6 +419,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
                     // ---- usage inside the window: parent's profile (or the usage carried across the
                     // inserted step) plus the corrections
                     const int32_t L = hi_w - lo_w + 1;
+                    out_win = max(L, 0);
                     MemT cross = 0;
                     if (ji != kEditNone) {
                         if (ji + 1 < Tc) {
@@ -462,6 +464,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
             p.out_peak[e] = out_pk;
             p.out_dur[e] = out_du;
             p.out_status[e] = out_st;
+            if (p.out_window) p.out_window[e] = out_win;
         }
         __syncwarp();
     }

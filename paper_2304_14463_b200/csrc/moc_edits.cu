@@ -132,7 +132,8 @@ int moc_cache_build(moc_cache* h, const int32_t* seqs, const int32_t* lens, int3
 }
 
 int moc_eval_edits(const moc_cache* h, const int32_t* parent, const int32_t* op, const int32_t* q, const int32_t* j,
-                   int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_status, void* stream) {
+                   int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_status, int32_t* out_window,
+                   void* stream) {
     clear_error();
     launch_counter() = 0;
     if (!h || B < 0) return fail(MOC_ERR_ARG, "moc_eval_edits: null handle or B < 0");
@@ -152,6 +153,7 @@ int moc_eval_edits(const moc_cache* h, const int32_t* parent, const int32_t* op,
     p.out_peak = out_peak;
     p.out_dur = out_dur;
     p.out_status = out_status;
+    p.out_window = out_window;
     const size_t msz = h->wide ? 8 : 4;
     const size_t warp_b = 2 * ((((size_t)h->c.stride + 4) * msz + 15) & ~size_t(15));
     p.warp_bytes = (uint32_t)warp_b;
