@@ -434,6 +434,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
             pred_start.assign((size_t)n + 1, 0);
             pred.resize((size_t)std::max<int64_t>(ne, 1));
             for (int64_t k = 0; k < ne; ++k) pred_start[(keys[k] & 0xFFFFFFFFu) + 1]++;
+            for (int32_t v = 0; v < n; ++v) g->max_indeg = std::max(g->max_indeg, pred_start[v + 1]);
             for (int32_t v = 0; v < n; ++v) pred_start[v + 1] += pred_start[v];
             std::vector<int32_t> fill(pred_start.begin(), pred_start.end() - 1);
             for (int64_t k = 0; k < ne; ++k) pred[fill[keys[k] & 0xFFFFFFFFu]++] = (int32_t)(keys[k] >> 32);

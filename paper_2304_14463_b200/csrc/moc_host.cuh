@@ -73,6 +73,7 @@ struct moc_graph {
     int32_t* d_pred_start = nullptr;     // predecessor lists (CSR), for the incremental evaluation
     int32_t* d_pred = nullptr;
     int64_t sink_m = 0;                   // sum of m over the nodes without successors
+    int32_t max_indeg = 0;                // largest number of predecessors of a node
     int64_t* d_w = nullptr;
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;
