@@ -121,18 +121,19 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         const int pre = n < 256 ? 0 : (int)std::min<int64_t>(5, (n * 13 / 10 + 96) / 128);
         PairFn fn = pair_fn(pl.wide, pre);
         int best_wpb = 0, best_warps = 0, best_nb = 0;
-        const int cand[4] = {16, 12, 8, 4};
-        const int max_wpb = pre > 0 ? 12 : 16;   // the look-ahead variants are compiled for at most 384 threads
-        for (int ci = 0; ci < 4; ++ci) {
-            const int wpb = std::min(g->want_gpc ? g->want_gpc : cand[ci], max_wpb);
+        if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) cudaGetLastError();
+        for (int wpb = 16; wpb >= 4; --wpb) {    // every kernel variant is compiled for up to 512 threads, two blocks per SM
+            if (g->want_gpc && wpb != std::min(g->want_gpc, 16)) continue;
             const size_t sm = graph_b + wpb * warp_b;
-            if (sm > smem_cap) { if (g->want_gpc) break; else continue; }
-            if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (sm > smem_cap) continue;
             int nb = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, wpb * 32, sm) != cudaSuccess) { cudaGetLastError(); continue; }
+            pl.pair_nb[wpb] = nb;
             if (nb * wpb > best_warps) { best_warps = nb * wpb; best_wpb = wpb; best_nb = nb; }
-            if (g->want_gpc) break;
         }
+        pl.pair_graph_b = graph_b;
+        pl.pair_warp_b = warp_b;
+        pl.sm_count = g->sm_count;
         if (best_warps >= 8) {
             pl.pair = true;
             pl.pair_fn = fn;
@@ -241,7 +242,34 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
 int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_offs, const int32_t* seqs, const int32_t* lens,
                  int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
                  cudaStream_t st) {
-    const int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    int block = pl.block;
+    size_t smem = pl.smem;
+    if (pl.pair) {
+        // Shape of this launch.  A warp works through its sequences one after the other, so a launch
+        // takes ceil(sequences per block / warps per block) rounds, and a round costs about as much as
+        // the SM has warps (the kernel is bound by on-chip throughput) but never less than a round of a
+        // half-empty SM.  Pick the warps per block and blocks per SM with the least rounds x warps.
+        int64_t best_cost = INT64_MAX;
+        int best_w = pl.gpc, best_nb = std::max(1, pl.grid / std::max(1, pl.sm_count));
+        for (int wpb = 4; wpb <= 16; ++wpb) {
+            const int nb = pl.pair_nb[wpb];
+            if (nb < 1) continue;
+            const int64_t blocks = (int64_t)pl.sm_count * nb;
+            const int64_t per_block = (B + blocks - 1) / blocks;
+            const int64_t rounds = (per_block + wpb - 1) / wpb;
+            const int64_t cost = rounds * std::max(wpb * nb, 16);
+            // equal cost: fewer, larger blocks (every block stages the graph in its shared memory)
+            if (cost < best_cost || (cost == best_cost && nb <= best_nb)) {
+                best_cost = cost;
+                best_w = wpb;
+                best_nb = nb;
+            }
+        }
+        block = 32 * best_w;
+        smem = pl.pair_graph_b + (size_t)best_w * pl.pair_warp_b;
+        grid = (int)std::min<int64_t>((int64_t)pl.sm_count * best_nb, ((int64_t)B + best_w - 1) / best_w);
+    }
     if (offs && fill_offs) {
         moc::offsets_kernel<<<(B + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, B, offs);
         ++g_launches;
@@ -249,8 +277,8 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
     if (g->ev_before) MOC_CUDA(cudaEventRecord(g->ev_before, st));
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)pl.block);
-    cfg.dynamicSmemBytes = pl.smem;
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     if (pl.pair) {
         moc::PairParams q{};

@@ -27,6 +27,10 @@ struct Plan {
     bool pair = false;
     PairFn pair_fn = nullptr;
     uint32_t rec_bytes = 0, w_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
+    // blocks per SM the fast path reaches with 1..16 warps per block (0: does not fit), and its sizes
+    int pair_nb[17] = {0};
+    size_t pair_graph_b = 0, pair_warp_b = 0;
+    int sm_count = 0;
 };
 
 

@@ -116,10 +116,10 @@ template <> struct __align__(8) NodeRec<int32_t> { uint32_t nd; int32_t m; };
 template <> struct __align__(16) NodeRec<int64_t> { uint32_t nd; uint32_t pad; int64_t m; };
 
 // kPre: how many 16-byte vectors of the next row each lane fetches ahead (rows of about 128*kPre
-// steps; 0 for short rows, where the extra registers cost more than the wait).  With look-ahead the
-// block is at most 12 warps and the compiler may use the registers of two blocks per SM.
+// steps; 0 for short rows, where the extra registers cost more than the wait).  Blocks have up to 16
+// warps and two of them share an SM (62 registers per thread, no spills).
 template <typename MemT, int kPre>
-__global__ void __launch_bounds__(kPre > 0 ? 384 : 512, kPre > 0 ? 2 : 1) eval_pair_kernel(const PairParams p) {
+__global__ void __launch_bounds__(512, 2) eval_pair_kernel(const PairParams p) {
     extern __shared__ __align__(16) char smem[];
     __shared__ int64_t s_part[16];
     using Rec = NodeRec<MemT>;
