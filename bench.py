@@ -35,10 +35,10 @@ PCT = 80
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the evaluation kernel, from
 # one ncu capture with flushed caches (None when the kernel changed after the capture)
-NCU_TRAFFIC_BYTES = 34865920
+NCU_TRAFFIC_BYTES = 34867200
 # executed warp instructions of the same launch (smsp__inst_executed.sum of that capture)
-NCU_WARP_INSTRUCTIONS = 32496634
-NCU_TRAFFIC_SOURCE = "ncu --set full, one launch: dram read 34.86 MB, write 0 (the 0.33 MB of results were still in L2)"
+NCU_WARP_INSTRUCTIONS = 34807562
+NCU_TRAFFIC_SOURCE = "ncu --set full, one launch: dram read 34.87 MB, write 0 (the 0.33 MB of results were still in L2)"
 
 
 def load_peaks():
@@ -606,7 +606,7 @@ def main():
                          "kernel": "evaluation kernel (CUDA events around each launch, mean of %d)" % n_k,
                          "between_kernels_ms": float(np.mean(gap_ms)),
                          "note": "the kernel is bound by shared-memory wavefronts and instruction issue, "
-                                 "not by HBM (ncu: issue slots 65 %, ALU pipe 55 %, shared-memory data pipe 64 %, DRAM 9 % busy)"},
+                                 "not by HBM (ncu: issue slots 71 %, ALU pipe 57 %, shared-memory data pipe 67 %, DRAM 9 % busy)"},
             "clocks": clocks.summary(),
         }
         if args.workload == WORKLOAD_IDX:
