@@ -66,6 +66,22 @@ def test_null_handles(binding):
     assert lib.moc_mem_profile(None, None, 0, None, None, None, None) == -1
     assert lib.moc_graph_set_launch(None, 0, 0) == -1
     assert lib.moc_last_error() != b""
+    # the later entry points: search, interval form, incremental evaluation
+    h = ctypes.c_void_p()
+    assert lib.moc_graph_set_node_caps(None, None) == -1
+    assert lib.moc_search_create(None, None, None, 1, 0, 0, 0, None, ctypes.byref(h)) == -1 and not h.value
+    assert lib.moc_search_run(None, 1, None) == -1
+    assert lib.moc_search_set_kinds(None, 7) == -1
+    assert lib.moc_search_state(None, None, None, None, None, None, None, None) == -1
+    assert lib.moc_search_best(None, None, None, None) == -1
+    assert lib.moc_search_info(None, None, None, None) == -1
+    lib.moc_search_destroy(None)
+    assert lib.moc_check_intervals(None, None, None, None, 1, 8, None, 0, None, None, None, None, None, None) == -1
+    assert lib.moc_cache_create(None, 1, ctypes.byref(h)) == -1 and not h.value
+    assert lib.moc_cache_build(None, None, None, 1, 0, None, None, None, None) == -1
+    assert lib.moc_eval_edits(None, None, None, None, None, 1, 0, None, None, None, None, None) == -1
+    lib.moc_cache_destroy(None)
+    assert b"moc_eval_edits" in lib.moc_last_error() or lib.moc_last_error() != b""
 
 
 def test_no_device_is_an_error_not_a_fallback(binding):
