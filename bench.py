@@ -564,14 +564,31 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- the same with 16-bit node ids on the host side (half the bytes over the host link)
+    e2e16_s, e2e16_steps = None, 0
+    if base.n <= 65535:
+        hr16 = [dict(r, seqs=torch.from_numpy(r["seqs"].numpy().astype(np.uint16)).pin_memory()) for r in hr]
+        for i in range(3):
+            r = hr16[i % len(hr16)]
+            G.eval_batch_host16(r["seqs"], r["lens"], M, r["peak"], r["dur"], r["st"])
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            r = hr16[i % len(hr16)]
+            G.eval_batch_host16(r["seqs"], r["lens"], M, r["peak"], r["dur"], r["st"])
+            e2e16_steps += r["steps"]
+        torch.cuda.synchronize()
+        e2e16_s = time.perf_counter() - t0
+
     # ---- max over ranks
     if world > 1:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device="cuda")
+        t = torch.tensor([ms, e2e_s, e2e16_s or 0.0], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms, e2e_s = float(t[0]), float(t[1])
-        tot = torch.tensor([steps_done, e2e_steps], dtype=torch.float64, device="cuda")
+        e2e16_s = float(t[2]) if e2e16_s is not None else None
+        tot = torch.tensor([steps_done, e2e_steps, e2e16_steps], dtype=torch.float64, device="cuda")
         dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-        steps_done, e2e_steps = float(tot[0]), float(tot[1])
+        steps_done, e2e_steps, e2e16_steps = float(tot[0]), float(tot[1]), float(tot[2])
 
     if rank == 0:
         peak_gbs, peak_kind = load_peaks()
@@ -597,6 +614,10 @@ def main():
             "e2e": {"value": e2e_steps / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": 4 * hr[0]["steps"] + 4 * hr[0]["B"], "d2h_bytes_per_step": 20 * hr[0]["B"],
                     "steps": n_e2e, "api": "moc_eval_batch_host (pinned host buffers)"},
+            "e2e_u16": None if e2e16_s is None else {
+                "value": e2e16_steps / e2e16_s, "unit": UNIT, "h2d_bytes_per_step": 2 * hr[0]["steps"] + 4 * hr[0]["B"],
+                "d2h_bytes_per_step": 20 * hr[0]["B"], "steps": n_e2e,
+                "api": "moc_eval_batch_host16 (node ids as uint16 in pinned host buffers)"},
             "roofline": {"bound": "hbm", "achieved": alg_bytes / (kernel_ms * 1e-3) / 1e9, "peak": peak_gbs,
                          "unit": "GB/s", "frac": alg_bytes / (kernel_ms * 1e-3) / 1e9 / peak_gbs,
                          "peak_kind": f"of {peak_kind}",

@@ -127,6 +127,16 @@ int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps
                         int64_t* out_dur, int32_t* out_feasible, void* stream);
 
 /*
+ * moc_eval_batch_host with the node ids as HOST uint16 (graphs with n <= 65535, else MOC_ERR_ARG):
+ * half the bytes cross the host link, which is what bounds the host entry point; the ids are widened
+ * on the device in front of the evaluation.  An id >= n is out of range as before (status -2).
+ * Everything else as moc_eval_batch_host.
+ */
+int moc_eval_batch_host16(const moc_graph* g, const uint16_t* seqs, int64_t n_steps,
+                          const int32_t* lens, int32_t B, int64_t M, int64_t* out_peak,
+                          int64_t* out_dur, int32_t* out_feasible, void* stream);
+
+/*
  * moc_eval_batch for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a deployment variant of moc_eval_batch, with identical results.)
  *

@@ -21,7 +21,7 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
            "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals",
-           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy"]
+           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy", "moc_eval_batch_host16"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -43,6 +43,8 @@ lib.moc_eval_batch.restype = ctypes.c_int
 lib.moc_eval_batch.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_eval_batch_host.restype = ctypes.c_int
 lib.moc_eval_batch_host.argtypes = [_P, _P, _i64, _P, _i32, _i64, _P, _P, _P, _P]
+lib.moc_eval_batch_host16.restype = ctypes.c_int
+lib.moc_eval_batch_host16.argtypes = [_P, _P, _i64, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_eval_batch_noalloc.restype = ctypes.c_int
 lib.moc_eval_batch_noalloc.argtypes = [_P, _P, _P, _i32, _i64, _P, _P, _P, _P]
 lib.moc_mem_profile.restype = ctypes.c_int
@@ -230,6 +232,17 @@ def moc_eval_batch_host(g, seqs, lens, M, out_peak, out_dur, out_feasible):
     return out_peak, out_dur, out_feasible
 
 
+def moc_eval_batch_host16(g, seqs, lens, M, out_peak, out_dur, out_feasible):
+    """moc_eval_batch_host with uint16 node ids (n <= 65535): half the bytes over the host link."""
+    import numpy as np
+    B = int(lens.shape[0])
+    rc = lib.moc_eval_batch_host16(g, _host(seqs, np.uint16, "seqs"), int(seqs.shape[0]), _host(lens, np.int32, "lens"),
+                                   B, int(M), _host(out_peak, np.int64, "out_peak"), _host(out_dur, np.int64, "out_dur"),
+                                   _host(out_feasible, np.int32, "out_feasible"), _stream())
+    _check(rc, "moc_eval_batch_host16")
+    return out_peak, out_dur, out_feasible
+
+
 def moc_mem_profile(g, seq, want_free=True):
     """One device sequence -> (profile[int64], free[int32] or None, status[int32 tensor of 1])."""
     import torch
@@ -369,6 +382,9 @@ class Graph:
 
     def eval_batch_host(self, seqs, lens, M, out_peak, out_dur, out_feasible):
         return moc_eval_batch_host(self.h, seqs, lens, M, out_peak, out_dur, out_feasible)
+
+    def eval_batch_host16(self, seqs, lens, M, out_peak, out_dur, out_feasible):
+        return moc_eval_batch_host16(self.h, seqs, lens, M, out_peak, out_dur, out_feasible)
 
     def mem_profile(self, seq, want_free=True):
         return moc_mem_profile(self.h, seq, want_free)

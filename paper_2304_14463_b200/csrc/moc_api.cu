@@ -680,6 +680,7 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_offs);
     cudaFree(g->d_state);
     cudaFree(g->d_stage_seqs);
+    cudaFree(g->d_stage_u16);
     cudaFree(g->d_stage_io);
     delete g;
 }
@@ -737,6 +738,50 @@ int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps
     MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, st));
     rc = launch_eval(g, g->d_stage_seqs, d_lens, B, M, d_peak, d_dur, d_st, st);
     if (rc != MOC_OK) return rc;
+    MOC_CUDA(cudaMemcpyAsync(out_peak, d_peak, bB * 8, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaMemcpyAsync(out_dur, d_dur, bB * 8, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaMemcpyAsync(out_feasible, d_st, bB * 4, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaStreamSynchronize(st));
+    return MOC_OK;
+}
+
+int moc_eval_batch_host16(const moc_graph* g, const uint16_t* seqs, int64_t n_steps, const int32_t* lens,
+                          int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur,
+                          int32_t* out_feasible, void* stream) {
+    g_err[0] = 0;
+    g_launches = 0;
+    if (!g || B < 0 || n_steps < 0) return fail(MOC_ERR_ARG, "moc_eval_batch_host16: null handle or negative size");
+    if (g->n > 65535) return fail(MOC_ERR_ARG, "moc_eval_batch_host16: n = %d does not fit 16-bit node ids", g->n);
+    if (B == 0) return MOC_OK;
+    if (!lens || !out_peak || !out_dur || !out_feasible || (n_steps > 0 && !seqs))
+        return fail(MOC_ERR_ARG, "moc_eval_batch_host16: null array");
+    int64_t need = 0;
+    for (int32_t b = 0; b < B; ++b) need += lens[b] > 0 ? lens[b] : 0;
+    if (need > n_steps) return fail(MOC_ERR_ARG, "moc_eval_batch_host16: lens sum to %lld > n_steps %lld", (long long)need, (long long)n_steps);
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = ensure((void**)&g->d_stage_seqs, &g->stage_seqs_cap, std::max<size_t>((size_t)need * 4, 16));
+    if (rc != MOC_OK) return rc;
+    rc = ensure((void**)&g->d_stage_u16, &g->stage_u16_cap, std::max<size_t>((size_t)need * 2, 16));
+    if (rc != MOC_OK) return rc;
+    const size_t bB = (size_t)B, o_lens = 0, o_peak = align16(bB * 4), o_dur = o_peak + bB * 8,
+                 o_st = o_dur + bB * 8, io_bytes = o_st + bB * 4;
+    rc = ensure((void**)&g->d_stage_io, &g->stage_io_cap, io_bytes);
+    if (rc != MOC_OK) return rc;
+    int32_t* d_lens = (int32_t*)(g->d_stage_io + o_lens);
+    int64_t* d_peak = (int64_t*)(g->d_stage_io + o_peak);
+    int64_t* d_dur = (int64_t*)(g->d_stage_io + o_dur);
+    int32_t* d_st = (int32_t*)(g->d_stage_io + o_st);
+    if (need) {
+        MOC_CUDA(cudaMemcpyAsync(g->d_stage_u16, seqs, (size_t)need * 2, cudaMemcpyHostToDevice, st));
+        const int blocks = (int)std::min<int64_t>((need / 8 + 255) / 256 + 1, (int64_t)g->sm_count * 8);
+        moc::widen_ids_kernel<<<blocks, 256, 0, st>>>(g->d_stage_u16, g->d_stage_seqs, need);
+    }
+    MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, st));
+    rc = launch_eval(g, g->d_stage_seqs, d_lens, B, M, d_peak, d_dur, d_st, st);
+    if (rc != MOC_OK) return rc;
+    if (need) ++g_launches;
     MOC_CUDA(cudaMemcpyAsync(out_peak, d_peak, bB * 8, cudaMemcpyDeviceToHost, st));
     MOC_CUDA(cudaMemcpyAsync(out_dur, d_dur, bB * 8, cudaMemcpyDeviceToHost, st));
     MOC_CUDA(cudaMemcpyAsync(out_feasible, d_st, bB * 4, cudaMemcpyDeviceToHost, st));

@@ -102,6 +102,8 @@ struct moc_graph {
     mutable size_t state_cap = 0;
     mutable int32_t* d_stage_seqs = nullptr;
     mutable size_t stage_seqs_cap = 0;
+    mutable uint16_t* d_stage_u16 = nullptr;   // 16-bit node ids as they arrive from the host
+    mutable size_t stage_u16_cap = 0;
     mutable char* d_stage_io = nullptr;  // lens | peak | dur | status
     mutable size_t stage_io_cap = 0;
 };

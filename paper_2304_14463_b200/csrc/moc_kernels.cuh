@@ -410,4 +410,23 @@ static __global__ void __launch_bounds__(kOffsThreads) offsets_kernel(const int3
     }
 }
 
+// 16-bit node ids -> 32-bit node ids (the evaluation kernels read int32 rows); 8 ids per thread and
+// step through 16-byte loads when the source is aligned.
+static __global__ void __launch_bounds__(256) widen_ids_kernel(const uint16_t* __restrict__ src, int32_t* __restrict__ dst, int64_t count) {
+    const int64_t n8 = count >> 3, stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((reinterpret_cast<uintptr_t>(src) & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        const uint4* s4 = reinterpret_cast<const uint4*>(src);
+        int4* d4 = reinterpret_cast<int4*>(dst);
+        for (int64_t i = tid; i < n8; i += stride) {
+            const uint4 v = __ldg(s4 + i);
+            d4[2 * i] = make_int4((int)(v.x & 0xFFFFu), (int)(v.x >> 16), (int)(v.y & 0xFFFFu), (int)(v.y >> 16));
+            d4[2 * i + 1] = make_int4((int)(v.z & 0xFFFFu), (int)(v.z >> 16), (int)(v.w & 0xFFFFu), (int)(v.w >> 16));
+        }
+        for (int64_t i = 8 * n8 + tid; i < count; i += stride) dst[i] = (int32_t)src[i];
+    } else {
+        for (int64_t i = tid; i < count; i += stride) dst[i] = (int32_t)src[i];
+    }
+}
+
 }  // namespace moc

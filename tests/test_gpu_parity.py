@@ -300,6 +300,32 @@ def test_host_entry_point(B):
     assert (p2 == op).all() and (d2 == od).all() and (s2 == os_).all()
 
 
+def test_host_entry_point_u16(B):
+    """16-bit node ids from the host: same results, ids >= n stay out of range, odd lengths and tails."""
+    wl = W.make(2, seed=4, B=777)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=2, frac=1 / 8)
+    seqs = np.where(seqs < 0, 65535, seqs).astype(np.int32)          # what 16 bits can carry of a damaged id
+    M = O.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    op, od, os_, _ = O.eval_batch(seqs, lens, M)
+    s16 = torch.from_numpy(seqs.astype(np.uint16)).pin_memory()
+    l = torch.from_numpy(lens).pin_memory()
+    peak = torch.empty(len(lens), dtype=torch.int64).pin_memory()
+    dur = torch.empty(len(lens), dtype=torch.int64).pin_memory()
+    st = torch.empty(len(lens), dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        G.eval_batch_host16(s16, l, M, peak, dur, st)
+        assert (peak.numpy() == op).all() and (dur.numpy() == od).all() and (st.numpy() == os_).all()
+    assert (os_ == -2).any() and (os_ >= 0).any()
+    # pageable, unaligned source
+    buf = np.zeros(len(seqs) + 1, np.uint16)
+    buf[1:] = seqs
+    p2, d2, s2 = np.empty(len(lens), np.int64), np.empty(len(lens), np.int64), np.empty(len(lens), np.int32)
+    G.eval_batch_host16(buf[1:], lens, M, p2, d2, s2)
+    assert (p2 == op).all() and (d2 == od).all() and (s2 == os_).all()
+
+
 def test_state_in_global_memory(B):
     """A graph whose per-sequence state exceeds shared memory (and > 65534 steps per sequence)."""
     n, C = 40000, 2
