@@ -542,6 +542,28 @@ def main():
     kern_ms = np.array([a.elapsed_time(b) for a, b in evs])
     gap_ms = np.array([evs[i][1].elapsed_time(evs[i + 1][0]) for i in range(n_k - 1)]) if n_k > 1 else np.zeros(1)
 
+    # ---- the same steps replayed from one CUDA graph: what is left when the host's launch path is taken out
+    graph_ms = None
+    try:
+        n_g = min(len(ring) * 4, 64)
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg):
+            for i in range(n_g):
+                step(i)
+        cg.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(1, args.steps // n_g)
+        g0.record()
+        for _ in range(reps):
+            cg.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / (reps * n_g)
+    except Exception as ex:                       # capture is a measurement aid, never a requirement
+        graph_ms = None
+        print(f"# CUDA graph capture skipped: {ex}", file=sys.stderr)
+
     # ---- end to end: host buffers in, host buffers out, through the host entry point
     hr = []
     for seqs, lens in ring_host[:4]:
@@ -626,6 +648,7 @@ def main():
                          "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": kernel_ms,
                          "kernel": "evaluation kernel (CUDA events around each launch, mean of %d)" % n_k,
                          "between_kernels_ms": float(np.mean(gap_ms)),
+                         "graph_replay_ms_per_step": graph_ms,
                          "note": "the kernel is bound by shared-memory wavefronts and instruction issue, "
                                  "not by HBM (ncu: issue slots 71 %, ALU pipe 57 %, shared-memory data pipe 67 %, DRAM 9 % busy)"},
             "clocks": clocks.summary(),
