@@ -63,7 +63,7 @@ def load_library(path):
         lib.moc_oracle_accept.restype = i32
         lib.moc_oracle_accept.argtypes = [i64, i64, i32, i64, i64, i32, i64]
         lib.moc_oracle_search_run.restype = None
-        lib.moc_oracle_search_run.argtypes = [P, P, P, P, P, P, i32, i32, i64, u64, u32, u32, u32, u32, P]
+        lib.moc_oracle_search_run.argtypes = [P, P, P, P, P, P, i32, i32, i64, u64, u32, u32, u32, u32, u32, P]
         lib.moc_oracle_search_best.restype = i32
         lib.moc_oracle_search_best.argtypes = [P, P, P, i32, i64]
     return lib
@@ -199,13 +199,14 @@ def accept(child, parent, M, lib=None):
 class OracleSearch:
     """P chains of the search: rows of ``stride`` ints with lengths and evaluations."""
 
-    def __init__(self, graph: OracleGraph, seqs, lens, M, seed, stride=None, chain0=0, kinds=7):
+    def __init__(self, graph: OracleGraph, seqs, lens, M, seed, stride=None, chain0=0, kinds=7, samples=1):
         self.g = graph
         self._lib = graph._lib
         self.M = int(M)
         self.seed = int(seed)
         self.chain0 = int(chain0)
         self.kinds = int(kinds)
+        self.samples = int(samples)
         lens = np.ascontiguousarray(lens, dtype=np.int32)
         self.P = len(lens)
         self.stride = int(stride) if stride is not None else graph.C * graph.n
@@ -223,7 +224,7 @@ class OracleSearch:
         acc = np.zeros(1, np.int64)
         self._lib.moc_oracle_search_run(self.g._h, _ptr(self.pop), _ptr(self.lens), _ptr(self.peak),
                                         _ptr(self.dur), _ptr(self.status), self.P, self.stride, self.M,
-                                        self.seed, self.generation, int(n_gen), self.chain0, self.kinds, _ptr(acc))
+                                        self.seed, self.generation, int(n_gen), self.chain0, self.kinds, self.samples, _ptr(acc))
         self.generation += int(n_gen)
         self.accepted += int(acc[0])
         return int(acc[0])

@@ -29,6 +29,10 @@
  *     delete:  element q is removed                                                   (T-1 steps)
  *     move:    element q is removed, then inserted in front of index j = r2 mod T
  *              of the shortened sequence                                              (T steps)
+ * Several proposals per chain and generation ("samples" = E >= 1): proposal e = 0..E-1 uses counter
+ * (generation, chain, e, 0); the chain's candidate is the proposal with the smallest key among those
+ * with status >= 0 (the lowest e among equals), and it replaces the chain's sequence when it is not
+ * worse than it.  E = 1 is the single proposal described above.
  * A chain with T = 0 proposes nothing.  Proposals are judged by the evaluator alone: a length
  * outside [n, C*n], a node left without a copy or with more than C copies all give status -2
  * there, and such a proposal is refused.
@@ -123,39 +127,60 @@ int32_t moc_oracle_accept(int64_t peak_c, int64_t dur_c, int32_t st_c, int64_t p
  *           (the caller evaluates the initial population).
  *   chain0  global number of chain 0 (enters the random draws only).
  *   kinds   enabled kinds of edit (bit 0 insert, bit 1 delete, bit 2 move).
+ *   samples proposals per chain and generation (>= 1).
  *   n_accepted (may be NULL) receives the number of accepted proposals.
  */
 void moc_oracle_search_run(const void *g, int32_t *pop, int32_t *lens, int64_t *peak, int64_t *dur,
                            int32_t *status, int32_t P, int32_t stride, int64_t M, uint64_t seed,
-                           uint32_t gen0, uint32_t n_gen, uint32_t chain0, uint32_t kinds,
+                           uint32_t gen0, uint32_t n_gen, uint32_t chain0, uint32_t kinds, uint32_t samples,
                            int64_t *n_accepted) {
     int32_t *child = (int32_t *)malloc(((size_t)stride + 2) * sizeof(int32_t));
+    int32_t *cand = (int32_t *)malloc(((size_t)stride + 2) * sizeof(int32_t));
     const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
     int64_t acc = 0;
     for (uint32_t gen = gen0; gen < gen0 + n_gen; ++gen) {
         for (int32_t c = 0; c < P; ++c) {
             int32_t *row = pop + (size_t)c * stride;
             const int32_t T = lens[c];
-            const uint32_t ctr[4] = {gen, chain0 + (uint32_t)c, 0u, 0u};
-            uint32_t r[4];
-            moc_oracle_philox4x32_10(ctr, key, r);
-            const int32_t Tc = moc_oracle_mutate(row, T, r[0], r[1], r[2], kinds, child);
-            if (Tc < 0) continue;
-            int64_t pk, du;
-            int32_t st;
-            moc_oracle_eval(g, child, Tc, M, &pk, &du, &st, NULL, NULL);
-            if (!moc_oracle_accept(pk, du, st, peak[c], dur[c], status[c], M)) continue;
-            /* st >= 0 implies Tc <= C*n <= stride */
-            memcpy(row, child, (size_t)Tc * sizeof(int32_t));
-            lens[c] = Tc;
-            peak[c] = pk;
-            dur[c] = du;
-            status[c] = st;
+            /* the chain's candidate: best valid proposal of this generation */
+            int have = 0;
+            int32_t cand_T = 0, cand_st = -2;
+            int64_t cand_pk = -1, cand_du = -1;
+            for (uint32_t e = 0; e < samples; ++e) {
+                const uint32_t ctr[4] = {gen, chain0 + (uint32_t)c, e, 0u};
+                uint32_t r[4];
+                moc_oracle_philox4x32_10(ctr, key, r);
+                const int32_t Tc = moc_oracle_mutate(row, T, r[0], r[1], r[2], kinds, child);
+                if (Tc < 0) continue;
+                int64_t pk, du;
+                int32_t st;
+                moc_oracle_eval(g, child, Tc, M, &pk, &du, &st, NULL, NULL);
+                if (st < 0) continue;
+                /* strictly better than the candidate so far: the lowest e wins among equals */
+                if (!have || (moc_oracle_accept(pk, du, st, cand_pk, cand_du, cand_st, M) &&
+                              !moc_oracle_accept(cand_pk, cand_du, cand_st, pk, du, st, M))) {
+                    have = 1;
+                    cand_T = Tc;
+                    cand_pk = pk;
+                    cand_du = du;
+                    cand_st = st;
+                    memcpy(cand, child, (size_t)Tc * sizeof(int32_t));
+                }
+            }
+            if (!have) continue;
+            if (!moc_oracle_accept(cand_pk, cand_du, cand_st, peak[c], dur[c], status[c], M)) continue;
+            /* status >= 0 implies cand_T <= C*n <= stride */
+            memcpy(row, cand, (size_t)cand_T * sizeof(int32_t));
+            lens[c] = cand_T;
+            peak[c] = cand_pk;
+            dur[c] = cand_du;
+            status[c] = cand_st;
             ++acc;
         }
     }
     if (n_accepted) *n_accepted = acc;
     free(child);
+    free(cand);
 }
 
 /* Index of the best chain: smallest key (max(peak, M), duration), valid chains only, lowest index

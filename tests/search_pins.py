@@ -112,7 +112,7 @@ def _tiny_problem():
     return n, edges, w, m
 
 
-def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen, chain0=0, kinds=7):
+def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, gen0, n_gen, chain0=0, kinds=7, samples=1):
     """The generation loop restated in Python over the separately pinned pieces, with the
     set-definition evaluator of defs.py in place of the oracle's evaluator."""
     def ev(s):
@@ -123,13 +123,19 @@ def python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, ge
     key = [seed & 0xFFFFFFFF, seed >> 32]
     for gen in range(gen0, gen0 + n_gen):
         for c, r in enumerate(rows):
-            x = oracle.philox4x32_10([gen, chain0 + c, 0, 0], key, lib=lib)
-            child = list_edit(r, int(x[0]), int(x[1]), int(x[2]), kinds)
-            if child is None:
-                continue
-            e = ev(child)
-            if e[2] >= 0 and key_of(e, M) <= key_of(evs[c], M):
-                rows[c], evs[c] = child, e
+            best = None                                   # (key, e, child, evaluation): smallest key, then lowest e
+            for e_i in range(samples):
+                x = oracle.philox4x32_10([gen, chain0 + c, e_i, 0], key, lib=lib)
+                child = list_edit(r, int(x[0]), int(x[1]), int(x[2]), kinds)
+                if child is None:
+                    continue
+                e = ev(child)
+                if e[2] < 0:
+                    continue
+                if best is None or (key_of(e, M), e_i) < (best[0], best[1]):
+                    best = (key_of(e, M), e_i, child, e)
+            if best is not None and best[0] <= key_of(evs[c], M):
+                rows[c], evs[c] = best[2], best[3]
     return rows, evs
 
 
@@ -146,12 +152,13 @@ def pin_search_loop(make_graph, lib):
             lens = np.array([len(r) for r in rows], np.int32)
             chain0 = 0 if M == P0 else 1000
             kinds = 7 if seed == 1 else (4 if M == 1 else 6)
-            S = oracle.OracleSearch(g, seqs, lens, M, seed, chain0=chain0, kinds=kinds)
+            samples = 1 if M == P0 else (3 if seed == 1 else 5)
+            S = oracle.OracleSearch(g, seqs, lens, M, seed, chain0=chain0, kinds=kinds, samples=samples)
             done = 0
             for n_gen in (1, 7, 40):
                 before = [key_of((S.peak[c], S.dur[c], S.status[c]), M) for c in range(S.P)]
                 S.run(n_gen)
-                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen, chain0, kinds)
+                want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, M, seed, done, n_gen, chain0, kinds, samples)
                 done += n_gen
                 for c in range(S.P):
                     assert list(S.row(c)) == want_rows[c], (M, seed, c)
@@ -160,6 +167,26 @@ def pin_search_loop(make_graph, lib):
                     assert after <= before[c]                     # the key never increases
                 rows = want_rows
             assert S.generation == done
+
+
+def pin_sample_ties(make_graph, lib):
+    """Four nodes without edges: every order has the same peak and duration, so all samples of a
+    generation tie and the first one (e = 0) must be taken."""
+    n, edges, w, m, C = 4, [], [1, 2, 3, 4], [5, 5, 5, 5], 2
+    g = make_graph(n, edges, w, m, C)
+    rows = [[0, 1, 2, 3], [3, 2, 1, 0], [1, 0, 3, 2]]
+    seqs = np.array([x for r in rows for x in r], np.int32)
+    lens = np.array([len(r) for r in rows], np.int32)
+    S = oracle.OracleSearch(g, seqs, lens, 100, seed=5, kinds=4, samples=4)
+    S.run(12)
+    want_rows, want_ev = python_generation_loop(make_graph, lib, n, edges, w, m, C, rows, 100, 5, 0, 12, 0, 4, 4)
+    for c in range(3):
+        assert list(S.row(c)) == want_rows[c], c
+    # the same draws with one sample take the e = 0 proposal too
+    S1 = oracle.OracleSearch(g, seqs, lens, 100, seed=5, kinds=4, samples=1)
+    S1.run(12)
+    for c in range(3):
+        assert list(S1.row(c)) == list(S.row(c))
 
 
 def pin_search_reaches_optimum(make_graph, lib):
@@ -214,4 +241,5 @@ def run_all(make_graph, lib):
     pin_edits(lib)
     pin_accept(lib)
     pin_search_loop(make_graph, lib)
+    pin_sample_ties(make_graph, lib)
     pin_search_reaches_optimum(make_graph, lib)

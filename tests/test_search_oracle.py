@@ -33,10 +33,13 @@ MUTANTS = {
     "accept_ignores_budget": ("const int64_t a = peak_c > M ? peak_c : M, b = peak_p > M ? peak_p : M;\n    if (a != b) return a < b;\n    return dur_c",
                               "const int64_t a = peak_c, b = peak_p;\n    if (a != b) return a < b;\n    return dur_c"),
     "accept_invalid_child": ("if (st_c < 0) return 0;", "if (st_c < -1) return 0;"),
-    "counter_transposed": ("{gen, chain0 + (uint32_t)c, 0u, 0u}", "{chain0 + (uint32_t)c, gen, 0u, 0u}"),
-    "chain_offset_ignored": ("{gen, chain0 + (uint32_t)c, 0u, 0u}", "{gen, (uint32_t)c, 0u, 0u}"),
+    "counter_transposed": ("{gen, chain0 + (uint32_t)c, e, 0u}", "{chain0 + (uint32_t)c, gen, e, 0u}"),
+    "chain_offset_ignored": ("{gen, chain0 + (uint32_t)c, e, 0u}", "{gen, (uint32_t)c, e, 0u}"),
+    "sample_not_in_counter": ("{gen, chain0 + (uint32_t)c, e, 0u}", "{gen, chain0 + (uint32_t)c, 0u, e}"),
+    "last_sample_wins_ties": ("                              !moc_oracle_accept(cand_pk, cand_du, cand_st, pk, du, st, M))) {", "                              1)) {"),
+    "first_valid_sample_taken": ("if (!have || (moc_oracle_accept(pk, du, st, cand_pk, cand_du, cand_st, M) &&", "if (!have || (0 &&"),
     "key_halves_swapped": ("{(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)}", "{(uint32_t)(seed >> 32), (uint32_t)(seed & 0xFFFFFFFFu)}"),
-    "fitness_not_updated": ("dur[c] = du;\n", ""),
+    "fitness_not_updated": ("dur[c] = cand_du;\n", ""),
     "best_last_of_equals": ("(a == b && dur[c] < dur[best])", "(a == b && dur[c] <= dur[best])"),
 }
 
