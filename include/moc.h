@@ -342,6 +342,23 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream);
 int moc_search_set_kinds(moc_search* s, uint32_t kinds);
 
 /*
+ * Proposals per chain and generation, and how they are scored.
+ *   samples      E >= 1.  Proposal e = 0..E-1 of chain c in generation k draws
+ *                Philox4x32-10(counter = (k, first_chain + c, e, 0)); the chain's candidate is the
+ *                proposal with the smallest key among those with status >= 0, the lowest e among
+ *                equals, and it replaces the chain's sequence when its key is not larger.  E = 1 is
+ *                the single proposal described above.
+ *   incremental  0: every proposal is written out and evaluated from scratch (E must be 1);
+ *                1: proposals are scored from the cached evaluation of the chain's sequence
+ *                (moc_eval_edits) and only accepted ones are written out.  Needs C <= 2 and a valid
+ *                sequence (status >= 0) in every chain at the time of the call (MOC_ERR_ARG otherwise).
+ *                The two ways give identical chains.
+ * Synchronises the device, allocates (the cache of the chains, 28 bytes per proposal); after it
+ * moc_search_run allocates nothing.  With incremental = 1 a generation is four kernels.
+ */
+int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental);
+
+/*
  * Copies the chains' current state to DEVICE arrays of the caller (any pointer may be NULL):
  *   out_rows      P rows of `stride` ints (moc_search_info); row c holds chain c's sequence in its
  *                 first out_lens[c] entries, the rest of the row is left untouched;

@@ -21,7 +21,7 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
            "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals",
-           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy", "moc_eval_batch_host16"]
+           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy", "moc_eval_batch_host16", "moc_search_set_samples"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -69,6 +69,8 @@ lib.moc_search_run.restype = ctypes.c_int
 lib.moc_search_run.argtypes = [_P, _i32, _P]
 lib.moc_search_set_kinds.restype = ctypes.c_int
 lib.moc_search_set_kinds.argtypes = [_P, ctypes.c_uint32]
+lib.moc_search_set_samples.restype = ctypes.c_int
+lib.moc_search_set_samples.argtypes = [_P, _i32, _i32]
 lib.moc_search_state.restype = ctypes.c_int
 lib.moc_search_state.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P]
 lib.moc_search_best.restype = ctypes.c_int
@@ -427,6 +429,10 @@ class Search:
 
     def set_kinds(self, kinds):
         moc_search_set_kinds(self.h, kinds)
+
+    def set_samples(self, samples, incremental=True):
+        """samples proposals per chain and generation; incremental: scored from the cached evaluation."""
+        _check(lib.moc_search_set_samples(self.h, int(samples), 1 if incremental else 0), "moc_search_set_samples")
 
     def info(self):
         return moc_search_info(self.h)

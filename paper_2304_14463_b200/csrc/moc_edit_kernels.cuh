@@ -55,6 +55,8 @@ struct PrepParams {
     int64_t* out_peak;          // may be null
     int64_t* out_dur;
     int32_t* out_status;
+    const int32_t* todo;        // may be null: indices of the parents to (re)build, todo_count of them
+    const int32_t* todo_count;  // device counter read by the kernel
     uint32_t warp_bytes;
 };
 
@@ -120,7 +122,9 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
     const int32_t n = c.n;
     constexpr uint32_t kFull = 0xFFFFFFFFu;
 
-    for (int32_t b = blockIdx.x * wpb + warp; b < c.P; b += gridDim.x * wpb) {
+    const int32_t count = p.todo != nullptr ? min(*p.todo_count, c.P) : c.P;
+    for (int32_t it = blockIdx.x * wpb + warp; it < count; it += gridDim.x * wpb) {
+        const int32_t b = p.todo != nullptr ? p.todo[it] : it;
         const int32_t T = p.lens[b];
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;

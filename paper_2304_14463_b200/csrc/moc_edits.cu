@@ -3,26 +3,40 @@
 #include <algorithm>
 #include <new>
 
-#include "moc_host.cuh"
-#include "moc_edit_kernels.cuh"
+#include "moc_cache_host.cuh"
 
 using namespace moc_host;
-
-struct moc_cache {
-    const moc_graph* g = nullptr;
-    int device = 0;
-    int32_t max_parents = 0;
-    bool wide = false;
-    char* d_block = nullptr;
-    int64_t* d_offs = nullptr;     // max_parents + 1
-    moc::EditCacheDev c{};
-    size_t warp_bytes = 0;
-    int wpb = 0, grid_cap = 0;
-};
 
 namespace {
 size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 }  // namespace
+
+namespace moc_host {
+int cache_prepare(moc_cache* h, const int32_t* seqs, const int32_t* lens, const int64_t* offs, int32_t P,
+                  const int32_t* todo, const int32_t* todo_count, int64_t M, int64_t* out_peak, int64_t* out_dur,
+                  int32_t* out_status, cudaStream_t st) {
+    h->c.P = P;
+    h->c.cap = h->g->d_cap;
+    moc::PrepParams p{};
+    p.c = h->c;
+    p.seqs = seqs;
+    p.lens = lens;
+    p.offs = offs;
+    p.M = M;
+    p.out_peak = out_peak;
+    p.out_dur = out_dur;
+    p.out_status = out_status;
+    p.todo = todo;
+    p.todo_count = todo_count;
+    p.warp_bytes = (uint32_t)h->warp_bytes;
+    auto fn = h->wide ? moc::edit_prepare_kernel<int64_t> : moc::edit_prepare_kernel<int32_t>;
+    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
+    const int grid = (int)std::min<int64_t>(h->grid_cap, ((int64_t)P + h->wpb - 1) / h->wpb);
+    fn<<<grid, 32 * h->wpb, h->warp_bytes * h->wpb, st>>>(p);
+    MOC_CUDA(cudaGetLastError());
+    return MOC_OK;
+}
+}  // namespace moc_host
 
 extern "C" {
 
@@ -109,24 +123,9 @@ int moc_cache_build(moc_cache* h, const int32_t* seqs, const int32_t* lens, int3
     DeviceGuard dg(h->device);
     if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", h->device);
     cudaStream_t st = (cudaStream_t)stream;
-    h->c.P = P;
-    h->c.cap = h->g->d_cap;
-    moc::PrepParams p{};
-    p.c = h->c;
-    p.seqs = seqs;
-    p.lens = lens;
-    p.offs = h->d_offs;
-    p.M = M;
-    p.out_peak = out_peak;
-    p.out_dur = out_dur;
-    p.out_status = out_status;
-    p.warp_bytes = (uint32_t)h->warp_bytes;
     moc::offsets_kernel<<<(P + moc::kOffsTile - 1) / moc::kOffsTile, moc::kOffsThreads, 0, st>>>(lens, P, h->d_offs);
-    auto fn = h->wide ? moc::edit_prepare_kernel<int64_t> : moc::edit_prepare_kernel<int32_t>;
-    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
-    const int grid = (int)std::min<int64_t>(h->grid_cap, ((int64_t)P + h->wpb - 1) / h->wpb);
-    fn<<<grid, 32 * h->wpb, h->warp_bytes * h->wpb, st>>>(p);
-    MOC_CUDA(cudaGetLastError());
+    int rc = cache_prepare(h, seqs, lens, h->d_offs, P, nullptr, nullptr, M, out_peak, out_dur, out_status, st);
+    if (rc != MOC_OK) return rc;
     launch_counter() = 2;
     return MOC_OK;
 }

@@ -4,7 +4,9 @@
 #include <algorithm>
 #include <new>
 
-#include "moc_host.cuh"
+#include <vector>
+
+#include "moc_cache_host.cuh"
 #include "moc_search_kernels.cuh"
 
 using namespace moc_host;
@@ -19,6 +21,12 @@ struct moc_search {
     char* d_block = nullptr;   // one allocation, carved up below
     int32_t* d_bad = nullptr;
     moc::SearchParams p{};
+    // search on the incremental evaluation (off until moc_search_set_samples switches it on)
+    bool incremental = false;
+    int32_t samples = 1;
+    moc_cache* cache = nullptr;
+    char* d_inc = nullptr;
+    moc::SearchIncParams ip{};
 };
 
 namespace {
@@ -130,6 +138,26 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
     moc::SearchParams& p = s->p;
     const int blocks = chain_blocks(s->P);
     int launches = 0;
+    if (s->incremental) {
+        const int64_t nE = (int64_t)s->P * s->samples;
+        for (int32_t k = 0; k < n_generations; ++k) {
+            p.generation = s->generation + (uint32_t)k;
+            s->ip.s = p;
+            moc::search_draw_kernel<<<(unsigned)((nE + 255) / 256), 256, 0, st>>>(s->ip);
+            int rc = moc_eval_edits(s->cache, s->ip.e_parent, s->ip.e_op, s->ip.e_q, s->ip.e_j, (int32_t)nE, s->M,
+                                    s->ip.r_peak, s->ip.r_dur, s->ip.r_status, nullptr, stream);
+            if (rc != MOC_OK) return rc;
+            moc::search_pick_kernel<<<blocks, moc::kSearchThreads, 0, st>>>(s->ip);
+            rc = cache_prepare(s->cache, p.rows, p.lens, s->ip.row_offs, s->P, s->ip.todo, s->ip.todo_count, s->M,
+                               nullptr, nullptr, nullptr, st);
+            if (rc != MOC_OK) return rc;
+            launches += 4;
+        }
+        MOC_CUDA(cudaGetLastError());
+        s->generation += (uint32_t)n_generations;
+        launch_counter() = launches;
+        return MOC_OK;
+    }
     for (int32_t k = 0; k < n_generations; ++k) {
         p.generation = s->generation + (uint32_t)k;
         // settle the previous generation's proposals (none before the first one), propose the next
@@ -153,6 +181,71 @@ int moc_search_set_kinds(moc_search* s, uint32_t kinds) {
     clear_error();
     if (!s || kinds == 0 || kinds > 7u) return fail(MOC_ERR_ARG, "moc_search_set_kinds: null handle or mask outside 1..7");
     s->p.kinds = kinds;
+    return MOC_OK;
+}
+
+int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) {
+    clear_error();
+    if (!s || samples < 1 || samples > 4096 || (incremental != 0 && incremental != 1))
+        return fail(MOC_ERR_ARG, "moc_search_set_samples: null handle, samples outside [1, 4096] or flag outside {0, 1}");
+    if (samples > 1 && !incremental)
+        return fail(MOC_ERR_ARG, "moc_search_set_samples: more than one proposal per chain needs the incremental evaluation");
+    if ((int64_t)s->P * samples > INT32_MAX) return fail(MOC_ERR_ARG, "moc_search_set_samples: P * samples exceeds 2^31 - 1");
+    DeviceGuard dg(s->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", s->device);
+    MOC_CUDA(cudaDeviceSynchronize());          // generations in flight still use the old buffers
+    if (!incremental) {
+        s->incremental = false;
+        s->samples = 1;
+        return MOC_OK;
+    }
+    // every chain needs a valid evaluation to start from
+    std::vector<int32_t> st((size_t)s->P);
+    MOC_CUDA(cudaMemcpy(st.data(), s->p.status, (size_t)s->P * 4, cudaMemcpyDeviceToHost));
+    for (int32_t c = 0; c < s->P; ++c)
+        if (st[c] < 0)
+            return fail(MOC_ERR_ARG, "moc_search_set_samples: chain %d has no valid sequence (status %d); the incremental "
+                        "evaluation starts from valid sequences only", c, st[c]);
+    if (!s->cache) {
+        moc_cache* h = nullptr;
+        int rc = moc_cache_create(s->g, s->P, &h);
+        if (rc != MOC_OK) return rc;
+        s->cache = h;
+    }
+    const size_t nE = (size_t)s->P * samples, bP = (size_t)s->P;
+    const size_t o_par = 0, o_op = o_par + up256(nE * 4), o_q = o_op + up256(nE * 4), o_j = o_q + up256(nE * 4),
+                 o_st = o_j + up256(nE * 4), o_pk = o_st + up256(nE * 4), o_du = o_pk + up256(nE * 8),
+                 o_offs = o_du + up256(nE * 8), o_todo = o_offs + up256((bP + 1) * 8), o_cnt = o_todo + up256(bP * 4),
+                 total = o_cnt + 256;
+    if (s->d_inc) MOC_CUDA(cudaFree(s->d_inc));
+    s->d_inc = nullptr;
+    s->incremental = false;
+    cudaError_t e = cudaMalloc((void**)&s->d_inc, total);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, "moc_search_set_samples: %s", cudaGetErrorString(e));
+    }
+    char* b = s->d_inc;
+    moc::SearchIncParams& ip = s->ip;
+    ip.s = s->p;
+    ip.samples = samples;
+    ip.e_parent = (int32_t*)(b + o_par);
+    ip.e_op = (int32_t*)(b + o_op);
+    ip.e_q = (int32_t*)(b + o_q);
+    ip.e_j = (int32_t*)(b + o_j);
+    ip.r_status = (int32_t*)(b + o_st);
+    ip.r_peak = (int64_t*)(b + o_pk);
+    ip.r_dur = (int64_t*)(b + o_du);
+    ip.row_offs = (int64_t*)(b + o_offs);
+    ip.todo = (int32_t*)(b + o_todo);
+    ip.todo_count = (int32_t*)(b + o_cnt);
+    // cache of all chains from their current rows
+    moc::search_row_offsets_kernel<<<(s->P + 255) / 256, 256>>>(ip);
+    int rc = cache_prepare(s->cache, s->p.rows, s->p.lens, ip.row_offs, s->P, nullptr, nullptr, s->M, nullptr, nullptr, nullptr, nullptr);
+    if (rc != MOC_OK) return rc;
+    MOC_CUDA(cudaDeviceSynchronize());
+    s->samples = samples;
+    s->incremental = true;
     return MOC_OK;
 }
 
@@ -198,6 +291,8 @@ int moc_search_info(const moc_search* s, int32_t* P, int32_t* stride, uint32_t* 
 void moc_search_destroy(moc_search* s) {
     if (!s) return;
     DeviceGuard dg(s->device);
+    moc_cache_destroy(s->cache);
+    cudaFree(s->d_inc);
     cudaFree(s->d_block);
     delete s;
 }

@@ -73,6 +73,39 @@ __device__ __forceinline__ bool search_not_worse(int64_t pk_c, int64_t du_c, int
 
 constexpr int kSearchThreads = 256;  // 8 chains per block, one warp each
 
+// The (r0 mod k)-th enabled kind of edit, k = number of enabled kinds (order: insert, delete, move).
+__device__ __forceinline__ uint32_t search_pick_kind(uint32_t kinds, uint32_t r0) {
+    uint32_t pick = r0 % (uint32_t)__popc(kinds), op = 0;
+    for (uint32_t o = 0; o < 3; ++o) {
+        if (kinds >> o & 1u) {
+            if (pick == 0) { op = o; break; }
+            --pick;
+        }
+    }
+    return op;
+}
+
+// Writes the edited copy of src[0..T) to dst with the lanes of one warp: element qd taken out (none:
+// INT32_MAX), then x put in front of index j of what is left (none: INT32_MAX); Tc elements result.
+// 16-byte stores, sources through the read-only path.
+__device__ __forceinline__ void search_write_edited(const int32_t* __restrict__ src, int32_t* __restrict__ dst,
+                                                    int32_t Tc, int32_t qd, int32_t j, int32_t x, int lane) {
+    auto at = [&](int32_t i) -> int32_t {
+        if (i == j) return x;
+        const int32_t k = i - (i > j ? 1 : 0);       // index in the row without element qd
+        return __ldg(src + k + (k >= qd ? 1 : 0));
+    };
+    for (int32_t i0 = 4 * lane; i0 < Tc; i0 += 128) {
+        if (i0 + 4 <= Tc) {
+            int4 v;
+            v.x = at(i0); v.y = at(i0 + 1); v.z = at(i0 + 2); v.w = at(i0 + 3);
+            *reinterpret_cast<int4*>(dst + i0) = v;
+        } else {
+            for (int32_t i = i0; i < Tc; ++i) dst[i] = at(i);
+        }
+    }
+}
+
 // One warp per chain.  kSelect: settle the pending proposal of the chain (written by the previous
 // launch, scored since).  kPropose: write the next proposal.
 //   op = the (r0 mod k)-th of the k enabled kinds in the order insert (0), delete (1), move (2); r0 mod 3
@@ -117,15 +150,7 @@ __global__ void __launch_bounds__(kSearchThreads) search_step_kernel(const Searc
         return;
     }
     const uint4 r = philox4x32_10(make_uint4(p.generation, p.chain0 + (uint32_t)c, 0u, 0u), make_uint2(p.seed_lo, p.seed_hi));
-    // the (r0 mod k)-th enabled kind, k = number of enabled kinds
-    const uint32_t nk = (uint32_t)__popc(p.kinds);
-    uint32_t pick = r.x % nk, op = 0;
-    for (uint32_t o = 0; o < 3; ++o) {
-        if (p.kinds >> o & 1u) {
-            if (pick == 0) { op = o; break; }
-            --pick;
-        }
-    }
+    const uint32_t op = search_pick_kind(p.kinds, r.x);
     const int32_t q = (int32_t)(r.y % (uint32_t)T);
     // The proposal is "take element q out (delete, move), then put x in front of index j (insert,
     // move)"; qd / j beyond every index switch a half off.
@@ -138,21 +163,97 @@ __global__ void __launch_bounds__(kSearchThreads) search_step_kernel(const Searc
     const int32_t* __restrict__ src = p.rows + src_off;
     int32_t* __restrict__ dst = p.rows + dst_off;
     const int32_t x = __ldg(src + q);
-    // element i of the proposal: 16-byte stores, sources through the read-only path
-    auto at = [&](int32_t i) -> int32_t {
-        if (i == j) return x;
-        const int32_t k = i - (i > j ? 1 : 0);       // index in the row without element qd
-        return __ldg(src + k + (k >= qd ? 1 : 0));
-    };
-    for (int32_t i0 = 4 * lane; i0 < Tc; i0 += 128) {
-        if (i0 + 4 <= Tc) {
-            int4 v;
-            v.x = at(i0); v.y = at(i0 + 1); v.z = at(i0 + 2); v.w = at(i0 + 3);
-            *reinterpret_cast<int4*>(dst + i0) = v;
-        } else {
-            for (int32_t i = i0; i < Tc; ++i) dst[i] = at(i);
-        }
+    search_write_edited(src, dst, Tc, qd, j, x, lane);
+}
+
+// ---- search on the incremental evaluation: E proposals per chain and generation are drawn as edit
+// records, scored from the cached evaluation of the chain's sequence, and only the winner of a chain
+// is ever written out.
+struct SearchIncParams {
+    SearchParams s;
+    int32_t samples;        // E
+    int32_t* e_parent;      // P * E edit records: chain, kind, step, insertion index
+    int32_t* e_op;
+    int32_t* e_q;
+    int32_t* e_j;
+    int64_t* r_peak;        // P * E results of the incremental evaluation
+    int64_t* r_dur;
+    int32_t* r_status;
+    int64_t* row_offs;      // P + 1: offset of every chain's current row in `rows` (input of the cache build)
+    int32_t* todo;          // P: chains whose sequence changed in this generation
+    int32_t* todo_count;
+};
+
+// One thread per proposal: proposal e of chain c draws Philox4x32-10 with counter (generation, chain0 + c, e, 0).
+__global__ void __launch_bounds__(256) search_draw_kernel(const SearchIncParams p) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t == 0) *p.todo_count = 0;
+    if (t >= (int64_t)p.s.P * p.samples) return;
+    const int32_t c = (int32_t)(t / p.samples), e = (int32_t)(t % p.samples);
+    const int32_t T = p.s.lens[c];
+    const uint4 r = philox4x32_10(make_uint4(p.s.generation, p.s.chain0 + (uint32_t)c, (uint32_t)e, 0u),
+                                  make_uint2(p.s.seed_lo, p.s.seed_hi));
+    const uint32_t op = search_pick_kind(p.s.kinds, r.x);
+    const uint32_t Tu = (uint32_t)max(T, 1);
+    p.e_parent[t] = c;
+    p.e_op[t] = (int32_t)op;
+    p.e_q[t] = (int32_t)(r.y % Tu);
+    p.e_j[t] = op == 0 ? (int32_t)(r.z % (Tu + 1u)) : (int32_t)(r.z % Tu);
+}
+
+// One warp per chain: the best proposal of the chain (smallest key among status >= 0, lowest sample
+// among equals) replaces the chain's sequence when it is not worse; its row is written to the chain's
+// other row, and the chain is listed for the rebuild of its cache entry.
+__global__ void __launch_bounds__(kSearchThreads) search_pick_kernel(const SearchIncParams p) {
+    const SearchParams& s = p.s;
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * (kSearchThreads / 32) + (threadIdx.x >> 5);
+    if (c >= s.P) return;
+    constexpr uint32_t kFull = 0xFFFFFFFFu;
+    const int64_t kInf = INT64_MAX;
+    int64_t a = kInf, d = kInf;
+    int32_t be = INT32_MAX;
+    for (int32_t e = lane; e < p.samples; e += 32) {          // ascending e: ties keep the lowest sample
+        const int64_t i = (int64_t)c * p.samples + e;
+        if (p.r_status[i] < 0) continue;
+        const int64_t pk = p.r_peak[i], ca = pk > s.M ? pk : s.M, cd = p.r_dur[i];
+        if (ca < a || (ca == a && cd < d)) { a = ca; d = cd; be = e; }
     }
+    for (int o = 16; o > 0; o >>= 1) {
+        const int64_t a2 = __shfl_xor_sync(kFull, a, o), d2 = __shfl_xor_sync(kFull, d, o);
+        const int32_t e2 = __shfl_xor_sync(kFull, be, o);
+        if (a2 < a || (a2 == a && (d2 < d || (d2 == d && e2 < be)))) { a = a2; d = d2; be = e2; }
+    }
+    if (be == INT32_MAX) return;                                // no valid proposal
+    const int64_t i = (int64_t)c * p.samples + be;
+    const int64_t pk = p.r_peak[i], du = p.r_dur[i];
+    const int32_t st = p.r_status[i];
+    if (!search_not_worse(pk, du, st, s.peak[c], s.dur[c], s.status[c], s.M)) return;
+    const int32_t cur = s.cur[c], T = s.lens[c];
+    const int32_t op = p.e_op[i], q = p.e_q[i], j = p.e_j[i];
+    const int32_t qd = op >= 1 ? q : INT32_MAX, ji = op != 1 ? j : INT32_MAX;
+    const int32_t Tc = T + (op == 0 ? 1 : 0) - (op == 1 ? 1 : 0);
+    const int64_t src_off = ((int64_t)cur * s.P + c) * s.stride, dst_off = ((int64_t)(cur ^ 1) * s.P + c) * s.stride;
+    const int32_t x = __ldg(s.rows + src_off + q);
+    search_write_edited(s.rows + src_off, s.rows + dst_off, Tc, qd, ji, x, lane);
+    __syncwarp();
+    if (lane == 0) {
+        s.cur[c] = cur ^ 1;
+        s.lens[c] = Tc;
+        s.peak[c] = pk;
+        s.dur[c] = du;
+        s.status[c] = st;
+        s.n_acc[c] += 1;
+        p.row_offs[c] = dst_off;
+        p.todo[atomicAdd(p.todo_count, 1)] = c;
+    }
+}
+
+// Offsets of the chains' current rows, for the build of the whole cache.
+__global__ void search_row_offsets_kernel(const SearchIncParams p) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < p.s.P) p.row_offs[c] = ((int64_t)p.s.cur[c] * p.s.P + c) * p.s.stride;
+    if (c == 0) p.row_offs[p.s.P] = (int64_t)2 * p.s.P * p.s.stride;
 }
 
 // Start of a search: packed sequences (offs = exclusive prefix sum of the lengths) become rows

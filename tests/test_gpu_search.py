@@ -165,3 +165,55 @@ def test_search_full_size(B):
         S.run(g)
         OS.run(g)
         assert_state_equal(S, OS, f"full size after {OS.generation}")
+
+
+@pytest.mark.parametrize("idx,P,samples", [(0, 512, 1), (0, 512, 5), (1, 256, 4), (2, 256, 1), (2, 192, 16), (2, 64, 40)])
+def test_search_incremental_parity(B, idx, P, samples):
+    """Proposals scored from the cached evaluation (moc_search_set_samples): one or several per chain
+    and generation; every chain identical to the search oracle after each call."""
+    wl = W.make(idx, seed=3, B=P)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    S = B.Search(G, dev(wl.seqs), dev(wl.lens), M, 17)
+    S.set_samples(samples, incremental=True)
+    OS = OracleSearch(O, wl.seqs, wl.lens, M, 17, stride=S.info()["stride"], samples=samples)
+    for g in (1, 2, 25):
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"config {idx}, {samples} samples, after {OS.generation}")
+    assert OS.accepted > 0
+    if samples == 1:
+        # back to proposals evaluated from scratch, and forth again: same chains as the oracle throughout
+        S.set_samples(1, incremental=False)
+        S.run(7)
+        OS.run(7)
+        assert_state_equal(S, OS, "after switching to full evaluation")
+        S.set_samples(1, incremental=True)
+        S.run(7)
+        OS.run(7)
+        assert_state_equal(S, OS, "after switching back")
+
+
+def test_search_incremental_errors(B):
+    wl = W.make(1, seed=3, B=32)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs = wl.seqs.copy()
+    seqs[:wl.lens[0]] = seqs[:wl.lens[0]][::-1]            # chain 0 starts from an invalid order
+    S = B.Search(G, dev(seqs), dev(wl.lens), M, 1)
+    with pytest.raises(B.MocError) as e:
+        S.set_samples(4, incremental=True)
+    assert e.value.code == -1
+    with pytest.raises(B.MocError):
+        S.set_samples(4, incremental=False)                 # several samples need the incremental evaluation
+    with pytest.raises(B.MocError):
+        S.set_samples(0, incremental=True)
+    S.run(3)                                                # still usable in the old way
+    wl3 = W.make(3, seed=1, B=8)                            # C = 3: outside the incremental evaluation
+    G3 = B.Graph(wl3.n, wl3.edges, wl3.w, wl3.m, wl3.C)
+    S3 = B.Search(G3, dev(wl3.seqs), dev(wl3.lens), 1 << 60, 1)
+    with pytest.raises(B.MocError):
+        S3.set_samples(2, incremental=True)
