@@ -395,6 +395,27 @@ void moc_search_destroy(moc_search* s);
 int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t sequences_per_block);
 
 /*
+ * Which evaluation kernel moc_eval_batch uses, and in what shape.  The library has three families
+ * for the operation of Section 2 (Eqs. 1-8); all give the same results, and MOC_KERNEL_AUTO (the
+ * default) picks the fastest one that can serve the graph.  The call exists so that tests can
+ * compare every family with the oracle and so that launch shapes can be measured.
+ *   MOC_KERNEL_AUTO   a = b = 0.
+ *   MOC_KERNEL_GROUP  a group of a threads (0, 32 .. 1024) per sequence, b sequences per block
+ *                     (0 = choose); any C <= MOC_MAX_COPIES.  Same as moc_graph_set_launch(a, b).
+ *   MOC_KERNEL_WARP   one warp per sequence, b warps per block (0 or 4..16), a = 0; C <= 2.
+ *   MOC_KERNEL_LANE   one sequence per lane: a block keeps a group of a sequences (0, 8, 16, 32)
+ *                     on chip and its b warps (0 or an even number 2..32) share the work on them;
+ *                     C <= 2 and a graph whose state for a group fits in shared memory.
+ * MOC_ERR_ARG for an unknown kind or shape; a kind that cannot serve the graph with its current C
+ * is reported by the next moc_eval_batch (MOC_ERR_ARG), which evaluates nothing.
+ */
+#define MOC_KERNEL_AUTO 0
+#define MOC_KERNEL_GROUP 1
+#define MOC_KERNEL_WARP 2
+#define MOC_KERNEL_LANE 3
+int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b);
+
+/*
  * Measurement hook: while set, every moc_eval_batch on this handle records `before` right before
  * and `after` right after its evaluation kernel (the dominant kernel; the offsets kernel lies
  * outside the pair), on the stream of the call.  Both are cudaEvent_t created by the caller with

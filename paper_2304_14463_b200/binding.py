@@ -21,7 +21,8 @@ EXPORTS = ["moc_graph_create", "moc_graph_set_max_copies", "moc_graph_destroy", 
            "moc_last_launch_count", "moc_last_error", "moc_eval_batch_noalloc", "moc_graph_set_timing_events",
            "moc_search_create", "moc_search_run", "moc_search_state", "moc_search_best", "moc_search_info",
            "moc_search_destroy", "moc_search_set_kinds", "moc_graph_set_node_caps", "moc_check_intervals",
-           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy", "moc_eval_batch_host16", "moc_search_set_samples"]
+           "moc_cache_create", "moc_cache_build", "moc_eval_edits", "moc_cache_destroy", "moc_eval_batch_host16", "moc_search_set_samples",
+           "moc_graph_set_kernel"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2304_14463_b200.build` "
@@ -51,6 +52,8 @@ lib.moc_mem_profile.restype = ctypes.c_int
 lib.moc_mem_profile.argtypes = [_P, _P, _i32, _P, _P, _P, _P]
 lib.moc_graph_set_launch.restype = ctypes.c_int
 lib.moc_graph_set_launch.argtypes = [_P, _i32, _i32]
+lib.moc_graph_set_kernel.restype = ctypes.c_int
+lib.moc_graph_set_kernel.argtypes = [_P, _i32, _i32, _i32]
 lib.moc_graph_set_timing_events.restype = ctypes.c_int
 lib.moc_graph_set_timing_events.argtypes = [_P, _P, _P]
 lib.moc_check_intervals.restype = ctypes.c_int
@@ -165,6 +168,13 @@ def moc_graph_set_node_caps(g, caps):
 def moc_graph_set_launch(g, threads_per_sequence=0, sequences_per_block=0):
     _check(lib.moc_graph_set_launch(g, int(threads_per_sequence), int(sequences_per_block)),
            "moc_graph_set_launch")
+
+
+MOC_KERNEL_AUTO, MOC_KERNEL_GROUP, MOC_KERNEL_WARP, MOC_KERNEL_LANE = 0, 1, 2, 3
+
+
+def moc_graph_set_kernel(g, kind=MOC_KERNEL_AUTO, a=0, b=0):
+    _check(lib.moc_graph_set_kernel(g, int(kind), int(a), int(b)), "moc_graph_set_kernel")
 
 
 def moc_graph_set_timing_events(g, before=None, after=None):
@@ -378,6 +388,9 @@ class Graph:
 
     def set_launch(self, threads_per_sequence=0, sequences_per_block=0):
         moc_graph_set_launch(self.h, threads_per_sequence, sequences_per_block)
+
+    def set_kernel(self, kind=MOC_KERNEL_AUTO, a=0, b=0):
+        moc_graph_set_kernel(self.h, kind, a, b)
 
     def eval_batch(self, seqs, lens, M, **out):
         return moc_eval_batch(self.h, seqs, lens, M, **out)

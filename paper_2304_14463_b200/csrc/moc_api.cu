@@ -78,6 +78,25 @@ PairFn pair_fn_t(int pre) {
 }
 PairFn pair_fn(bool wide, int pre) { return wide ? pair_fn_t<int64_t>(pre) : pair_fn_t<int32_t>(pre); }
 
+template <typename MemT, int LG>
+LaneFn lane_fn_kp(int kp) {
+    switch (kp) {
+        case 2: return (LaneFn)moc::eval_lane_kernel<MemT, LG, 2>;
+        case 4: return (LaneFn)moc::eval_lane_kernel<MemT, LG, 4>;
+        case 6: return (LaneFn)moc::eval_lane_kernel<MemT, LG, 6>;
+        default: return (LaneFn)moc::eval_lane_kernel<MemT, LG, 8>;
+    }
+}
+template <typename MemT>
+LaneFn lane_fn_lg(int lg, int kp) {
+    switch (lg) {
+        case 5: return lane_fn_kp<MemT, 5>(kp);
+        case 4: return lane_fn_kp<MemT, 4>(kp);
+        default: return lane_fn_kp<MemT, 3>(kp);
+    }
+}
+LaneFn lane_fn(bool wide, int lg, int kp) { return wide ? lane_fn_lg<int64_t>(lg, kp) : lane_fn_lg<int32_t>(lg, kp); }
+
 // Raises a kernel's dynamic shared-memory limit to all the device offers beside its static part.
 cudaError_t raise_smem_limit(const void* fn, size_t smem_optin) {
     cudaFuncAttributes a{};
@@ -91,6 +110,61 @@ int pow2_ceil(int x) {
     int p = 1;
     while (p < x) p <<= 1;
     return p;
+}
+
+// Plan of the sequence-per-lane path: the largest group whose state fits beside the graph, with as
+// many warps per SM as fit.  Returns nullptr on success, else the reason it cannot serve the graph.
+const char* plan_lane(const moc_graph* g, size_t smem_cap, Plan* out) {
+    Plan pl = *out;
+    const int64_t n = g->n, C = g->C, t_max = C * n;
+    if (C > 2) return "C > 2";
+    if ((__int128)C * g->sum_w >= ((__int128)1 << 40)) return "C * sum(w) reaches 2^40";
+    const bool forced = g->want_kind == MOC_KERNEL_LANE;
+    const size_t msz = pl.wide ? 8 : 4;
+    for (int li = 0; li < 3; ++li) {
+        const int lg = 5 - li, gsz = 1 << lg, S = 32 >> lg;
+        const LaneLayout& L = g->lane[li];
+        if (!L.ok) continue;
+        if (forced && g->want_a && g->want_a != gsz) continue;
+        const size_t rec_b = 16 * (size_t)S * L.n_bundles, w_b = align16(8 * (size_t)S * L.n_bundles),
+                     succ_b = align16(4 * (size_t)L.succ_len), word_b = align16(4 * (size_t)gsz * (n + 3)),
+                     delta_b = align16(msz * gsz * (size_t)(t_max + 3));
+        int best_w = 0, best_nb = 0, best_kp = 0;
+        for (int w = 32; w >= 2; w -= 2) {
+            if (forced && g->want_b && g->want_b != w) continue;
+            const int Q = w * S;
+            const size_t sm = rec_b + w_b + succ_b + 2 * (size_t)Q * gsz * msz + word_b + delta_b;
+            if (sm > smem_cap) continue;
+            // vectors fetched ahead per sub-lane: enough for a typical row of about 1.3 n steps
+            int kp = (int)(((n * 13 / 10 + 6) / 4 + Q - 1) / Q);
+            kp = std::min(8, std::max(2, (kp + 1) & ~1));
+            LaneFn fn = lane_fn(pl.wide, lg, kp);
+            if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, w * 32, sm) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (nb < 1) continue;
+            // as many warps per SM as fit, up to 64; among equals the shape with more blocks
+            const int warps = std::min(nb * w, 64), best = std::min(best_nb * best_w, 64);
+            if (warps > best || (warps == best && nb > best_nb && w >= 8)) { best_w = w; best_nb = nb; best_kp = kp; }
+        }
+        if (best_w == 0) continue;
+        const int Q = best_w * S;
+        pl.lane = true;
+        pl.lane_fn = lane_fn(pl.wide, lg, best_kp);
+        pl.lane_lg = lg;
+        pl.G = 32 * best_w / gsz;
+        pl.gpc = gsz;
+        pl.block = 32 * best_w;
+        pl.smem = rec_b + w_b + succ_b + 2 * (size_t)Q * gsz * msz + word_b + delta_b;
+        pl.grid = g->sm_count * best_nb;
+        pl.sm_count = g->sm_count;
+        pl.lane_rec_b = (uint32_t)rec_b; pl.lane_w_b = (uint32_t)w_b; pl.lane_succ_b = (uint32_t)succ_b;
+        pl.lane_word_b = (uint32_t)word_b; pl.lane_delta_b = (uint32_t)delta_b;
+        pl.valid = true;
+        *out = pl;
+        return nullptr;
+    }
+    return "the state of a group of sequences exceeds shared memory in the requested shape, n >= 4096, or a degree above 255";
 }
 
 // Chooses kernel variant, group size and grid for the handle's current n and C.  The dynamic
@@ -107,7 +181,19 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
                  sh_delta = align16((t_max + 1) * mem_sz);
     const size_t sh_group = sh_cnt + sh_occ + sh_delta + align16(moc::kRedBytes);
     const size_t smem_cap = g->smem_optin > 1024 ? g->smem_optin - 1024 : 0;  // 1 KB per block is reserved
-    if (!profile && g->want_G == 0 && C <= 2 && g->d_rec32 != nullptr) {
+    const int kind = profile ? MOC_KERNEL_GROUP : g->want_kind;
+    const bool shape_given = g->want_G != 0 || g->want_gpc != 0;       // moc_graph_set_launch
+    if (kind == MOC_KERNEL_LANE || (kind == MOC_KERNEL_AUTO && !shape_given && !profile)) {
+        const char* why = plan_lane(g, smem_cap, &pl);
+        if (!why) {
+            *out = pl;
+            return MOC_OK;
+        }
+        if (kind == MOC_KERNEL_LANE) return fail(MOC_ERR_ARG, "the sequence-per-lane kernel cannot serve this graph: %s", why);
+    }
+    if (kind == MOC_KERNEL_WARP && (C > 2 || g->d_rec32 == nullptr))
+        return fail(MOC_ERR_ARG, "the warp-per-sequence kernel cannot serve this graph (C > 2 or degrees too uneven)");
+    if (!profile && g->want_G == 0 && kind != MOC_KERNEL_GROUP && C <= 2 && g->d_rec32 != nullptr) {
         // warp-per-sequence fast path
         const size_t msz = pl.wide ? 8 : 4, per_vec = 16 / msz;
         const size_t nvec_d = (t_max + 1 + per_vec - 1) / per_vec;
@@ -219,6 +305,95 @@ int ensure(void** ptr, size_t* cap, size_t need) {
     return MOC_OK;
 }
 
+
+// Durations of the sequence-per-lane layouts: w | 1 << 40 (counts the node when it has two copies)
+// | 1 << 52 when the node's cap C_v is 1.
+int upload_lane_w(moc_graph* g) {
+    for (int li = 0; li < 3; ++li) {
+        LaneLayout& L = g->lane[li];
+        if (!L.ok) continue;
+        std::vector<uint64_t> wx(L.h_node.size());
+        for (size_t r = 0; r < wx.size(); ++r) {
+            const int32_t v = L.h_node[r];
+            if (v < 0) { wx[r] = 0; continue; }
+            uint64_t x = (uint64_t)g->h_w[v] | (uint64_t(1) << moc::kLaneCntShift);
+            if (!g->h_cap.empty() && g->h_cap[v] == 1) x |= uint64_t(1) << moc::kLaneCapShift;
+            wx[r] = x;
+        }
+        MOC_CUDA(cudaMemcpy(L.d_w, wx.data(), wx.size() * 8, cudaMemcpyHostToDevice));
+    }
+    return MOC_OK;
+}
+
+// Layouts for the sequence-per-lane kernel, one per group size g = 32, 16, 8 (S = 1, 2, 4 sub-lanes).
+// Nodes in order of falling out-degree (a sink counts one: its made-up successor), S consecutive
+// nodes form a bundle and share a row count; entry (k, h) of a bundle is the byte offset of the
+// word row of the k-th successor of its h-th node, the node's own row once its list is used up.
+// Rows of the word array: 0..n-1 nodes, n spare (ids out of range), n+1 holds T, n+2 holds (1, 1).
+int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, const std::vector<int32_t>& succ,
+                       const int64_t* m, const std::vector<int32_t>& m32) {
+    const int32_t n = g->n;
+    if (n >= 4096) return MOC_OK;                       // the count of two-copy nodes has 12 bits
+    auto deg = [&](int32_t v) { return std::max(1, succ_start[v + 1] - succ_start[v]); };
+    std::vector<int32_t> order((size_t)n);
+    for (int32_t v = 0; v < n; ++v) order[v] = v;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
+    if (deg(order[0]) > 255) return MOC_OK;
+    for (int li = 0; li < 3; ++li) {
+        const int lg = 5 - li, gsz = 1 << lg, S = 32 >> lg;
+        LaneLayout& L = g->lane[li];
+        const int32_t nb = (n + S - 1) / S;
+        std::vector<int32_t> node((size_t)nb * S, -1);
+        for (int32_t i = 0; i < n; ++i) node[i] = order[i];
+        std::vector<uint4> rec32(node.size()), rec64(node.size());
+        std::vector<uint32_t> se;
+        const uint32_t row_b = 4u * (uint32_t)gsz;
+        for (int32_t bd = 0; bd < nb; ++bd) {
+            int rows = 0;
+            for (int h = 0; h < S; ++h)
+                if (node[(size_t)bd * S + h] >= 0) rows = std::max(rows, deg(node[(size_t)bd * S + h]));
+            const uint32_t first = (uint32_t)se.size();
+            for (int k = 0; k < rows; ++k)
+                for (int h = 0; h < S; ++h) {
+                    const int32_t v = node[(size_t)bd * S + h];
+                    uint32_t row;
+                    if (v < 0) row = (uint32_t)n + 2;
+                    else if (k < succ_start[v + 1] - succ_start[v]) row = (uint32_t)succ[succ_start[v] + k];
+                    else if (k == 0) row = (uint32_t)n + 1;          // a sink: the word that holds T
+                    else row = (uint32_t)v;
+                    se.push_back(row * row_b);
+                }
+            for (int h = 0; h < S; ++h) {
+                const size_t r = (size_t)bd * S + h;
+                const int32_t v = node[r];
+                const uint32_t x = (v >= 0 ? (uint32_t)v : (uint32_t)n + 2) * row_b;
+                const uint32_t y = (first + (uint32_t)h) | ((uint32_t)rows << 24);
+                const uint64_t mv = v >= 0 ? (uint64_t)m[v] : 0;
+                rec32[r] = make_uint4(x, y, v >= 0 ? (uint32_t)m32[v] : 0u, 0u);
+                rec64[r] = make_uint4(x, y, (uint32_t)(mv & 0xFFFFFFFFu), (uint32_t)(mv >> 32));
+            }
+        }
+        while (se.size() % 4) se.push_back(((uint32_t)n + 2) * row_b);
+        if (se.empty()) se.assign(4, ((uint32_t)n + 2) * row_b);
+        if (se.size() >= (size_t(1) << 24)) continue;
+        cudaError_t e = cudaMalloc(&L.d_rec32, rec32.size() * 16);
+        if (e == cudaSuccess) e = cudaMalloc(&L.d_rec64, rec64.size() * 16);
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L.d_w, align16(node.size() * 8));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L.d_succ, se.size() * 4);
+        if (e == cudaSuccess) e = cudaMemcpy(L.d_rec32, rec32.data(), rec32.size() * 16, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(L.d_rec64, rec64.data(), rec64.size() * 16, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemset(L.d_w, 0, align16(node.size() * 8));
+        if (e == cudaSuccess) e = cudaMemcpy(L.d_succ, se.data(), se.size() * 4, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess)
+            return fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, "moc_graph_create: %s", cudaGetErrorString(e));
+        L.n_bundles = nb;
+        L.succ_len = (int64_t)se.size();
+        L.h_node = node;
+        L.ok = true;
+    }
+    return upload_lane_w(g);
+}
+
 moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     moc::EvalParams p{};
     p.g.n = g->n;
@@ -242,7 +417,7 @@ moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
 int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_offs, const int32_t* seqs, const int32_t* lens,
                  int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
                  cudaStream_t st) {
-    int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);
+    int grid = (int)std::min<int64_t>(pl.grid, ((int64_t)B + pl.gpc - 1) / pl.gpc);   // lane path: gpc = sequences per group
     int block = pl.block;
     size_t smem = pl.smem;
     if (pl.pair) {
@@ -280,7 +455,28 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    if (pl.pair) {
+    if (pl.lane) {
+        const LaneLayout& L = g->lane[5 - pl.lane_lg];
+        moc::LaneParams q{};
+        q.n = g->n;
+        q.max_T = g->C * g->n;
+        q.B = B;
+        q.n_bundles = L.n_bundles;
+        q.M = M;
+        q.base_dur = g->sum_w;
+        q.rec = (const uint4*)(pl.wide ? L.d_rec64 : L.d_rec32);
+        q.wrec = L.d_w;
+        q.succ = L.d_succ;
+        q.seqs = seqs;
+        q.lens = lens;
+        q.offs = offs;
+        q.out_peak = out_peak;
+        q.out_dur = out_dur;
+        q.out_status = out_feasible;
+        q.rec_bytes = pl.lane_rec_b; q.w_bytes = pl.lane_w_b; q.succ_bytes = pl.lane_succ_b;
+        q.word_bytes = pl.lane_word_b; q.delta_bytes = pl.lane_delta_b;
+        MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.lane_fn, q));
+    } else if (pl.pair) {
         moc::PairParams q{};
         q.n = g->n;
         q.sell_len = g->sell_len;
@@ -325,7 +521,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
 // Each block of the self-addressing kernel re-reads the lengths in front of its range: worth it
 // while that redundant traffic (grid * B/2 * 4 bytes from L2) stays small next to a second launch.
 bool rows_without_scratch(const Plan& pl, int32_t B) {
-    return pl.pair && (int64_t)pl.grid * B * 2 <= (int64_t)16 << 20;
+    return (pl.pair || pl.lane) && (int64_t)pl.grid * B * 2 <= (int64_t)16 << 20;
 }
 
 int launch_eval(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B, int64_t M,
@@ -581,6 +777,16 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
         moc_graph_destroy(g);
         return rc;
     }
+    try {
+        rc = build_lane_layouts(g, succ_start, succ, m, m32);
+    } catch (const std::bad_alloc&) {
+        rc = fail(MOC_ERR_NOMEM, "host allocation failed");
+    }
+    if (rc != MOC_OK) {
+        cudaGetLastError();
+        moc_graph_destroy(g);
+        return rc;
+    }
     *out = g;
     return MOC_OK;
 }
@@ -638,7 +844,33 @@ int moc_graph_set_node_caps(moc_graph* g, const int32_t* caps) {
         MOC_CUDA(cudaFree(g->d_cap));
         g->d_cap = nullptr;
     }
-    return upload_wslot(g);
+    int rc = upload_wslot(g);
+    if (rc != MOC_OK) return rc;
+    return upload_lane_w(g);
+}
+
+int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b) {
+    g_err[0] = 0;
+    if (!g) return fail(MOC_ERR_ARG, "moc_graph_set_kernel: null handle");
+    bool ok = false;
+    switch (kind) {
+        case MOC_KERNEL_AUTO: ok = a == 0 && b == 0; break;
+        case MOC_KERNEL_GROUP:
+            ok = (a == 0 || a == 32 || a == 64 || a == 128 || a == 256 || a == 512 || a == 1024) && b >= 0 && b <= 32 &&
+                 !(a && b && a * b > 1024);
+            break;
+        case MOC_KERNEL_WARP: ok = a == 0 && (b == 0 || (b >= 4 && b <= 16)); break;
+        case MOC_KERNEL_LANE: ok = (a == 0 || a == 8 || a == 16 || a == 32) && (b == 0 || (b >= 2 && b <= 32 && b % 2 == 0)); break;
+        default: break;
+    }
+    if (!ok) return fail(MOC_ERR_ARG, "moc_graph_set_kernel: unsupported kind or shape (%d, %d, %d)", kind, a, b);
+    g->want_kind = kind;
+    g->want_a = a;
+    g->want_b = b;
+    g->want_G = kind == MOC_KERNEL_GROUP ? a : 0;
+    g->want_gpc = (kind == MOC_KERNEL_GROUP || kind == MOC_KERNEL_WARP) ? b : 0;
+    g->plan_eval.valid = false;
+    return MOC_OK;
 }
 
 int moc_graph_set_launch(moc_graph* g, int32_t tps, int32_t spb) {
@@ -646,6 +878,8 @@ int moc_graph_set_launch(moc_graph* g, int32_t tps, int32_t spb) {
     const bool ok_g = tps == 0 || tps == 32 || tps == 64 || tps == 128 || tps == 256 || tps == 512 || tps == 1024;
     if (!g || !ok_g || spb < 0 || spb > 32 || (tps && spb && tps * spb > 1024))
         return fail(MOC_ERR_ARG, "moc_graph_set_launch: unsupported shape (%d threads x %d sequences)", tps, spb);
+    g->want_kind = MOC_KERNEL_AUTO;
+    g->want_a = g->want_b = 0;
     g->want_G = tps;
     g->want_gpc = spb;
     g->plan_eval.valid = false;
@@ -682,6 +916,12 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_stage_seqs);
     cudaFree(g->d_stage_u16);
     cudaFree(g->d_stage_io);
+    for (int li = 0; li < 3; ++li) {
+        cudaFree(g->lane[li].d_rec32);
+        cudaFree(g->lane[li].d_rec64);
+        cudaFree(g->lane[li].d_w);
+        cudaFree(g->lane[li].d_succ);
+    }
     delete g;
 }
 

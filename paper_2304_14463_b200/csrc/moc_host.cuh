@@ -10,11 +10,13 @@
 #include "../../include/moc.h"
 #include "moc_kernels.cuh"
 #include "moc_pair_kernel.cuh"
+#include "moc_lane_kernel.cuh"
 
 namespace moc_host {
 
 using KernelFn = void (*)(const moc::EvalParams);
 using PairFn = void (*)(const moc::PairParams);
+using LaneFn = void (*)(const moc::LaneParams);
 
 struct Plan {
     bool valid = false;
@@ -31,6 +33,23 @@ struct Plan {
     int pair_nb[17] = {0};
     size_t pair_graph_b = 0, pair_warp_b = 0;
     int sm_count = 0;
+    // sequence-per-lane path for C <= 2: a block keeps a group of 8, 16 or 32 sequences on chip
+    bool lane = false;
+    LaneFn lane_fn = nullptr;
+    int lane_lg = 0;               // log2 of the sequences per group
+    uint32_t lane_rec_b = 0, lane_w_b = 0, lane_succ_b = 0, lane_word_b = 0, lane_delta_b = 0;
+};
+
+// Graph in the order the sequence-per-lane kernel walks it, for one group size (S = 32 / g sub-lanes).
+struct LaneLayout {
+    bool ok = false;
+    int32_t n_bundles = 0;
+    int64_t succ_len = 0;                 // entries of the successor array (a multiple of 4)
+    void* d_rec32 = nullptr;              // uint4 records with 32-bit / 64-bit output sizes
+    void* d_rec64 = nullptr;
+    uint64_t* d_w = nullptr;
+    uint32_t* d_succ = nullptr;
+    std::vector<int32_t> h_node;          // node of every slot (-1: none)
 };
 
 
@@ -82,6 +101,8 @@ struct moc_graph {
     int64_t* d_m64 = nullptr;
     int32_t* d_m32 = nullptr;
     int32_t want_G = 0, want_gpc = 0;
+    int32_t want_kind = 0, want_a = 0, want_b = 0;   // moc_graph_set_kernel
+    moc_host::LaneLayout lane[3];         // groups of 32, 16, 8 sequences
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
     // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
     int32_t sell_len = 0, n_tiles = 0;

@@ -65,6 +65,7 @@ def test_null_handles(binding):
     assert lib.moc_eval_batch(None, None, None, 0, 0, None, None, None, None) == -1
     assert lib.moc_mem_profile(None, None, 0, None, None, None, None) == -1
     assert lib.moc_graph_set_launch(None, 0, 0) == -1
+    assert lib.moc_graph_set_kernel(None, 0, 0, 0) == -1
     assert lib.moc_last_error() != b""
     # the later entry points: search, interval form, incremental evaluation
     h = ctypes.c_void_p()

@@ -126,6 +126,51 @@ def test_mem_profile_parity(B, idx):
     assert free is None and (prof.cpu().numpy() == r["profile"]).all()
 
 
+# ------------------------------------------------------------------ every kernel family
+LANE_SHAPES = [(0, 0), (32, 32), (32, 16), (32, 6), (16, 32), (16, 12), (16, 2), (8, 32), (8, 10)]
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+@pytest.mark.parametrize("a,b", LANE_SHAPES)
+def test_lane_kernel_shapes(B, idx, a, b):
+    """The sequence-per-lane kernel in every group size and with few and many warps: damaged batches of
+    the three configurations it serves, a batch size that leaves the last group ragged."""
+    wl = W.make(idx, seed=7, B=[333, 1500, 777][idx])
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    try:
+        G.set_kernel(B.MOC_KERNEL_LANE, a, b)
+        seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=5, frac=1 / 8)
+        peaks = O.eval_batch(seqs, lens, BIG)[0]
+        assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), f"lane {a}x{b} {wl.name}")
+    except B.MocError as ex:
+        # only shapes whose group state exceeds shared memory may be refused
+        assert "cannot serve" in str(ex) and idx == 2 and a == 32 and b > 16, str(ex)
+
+
+@pytest.mark.parametrize("kind", ["group", "warp", "lane"])
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_kernel_families_agree_with_oracle(B, idx, kind):
+    """Each family forced in turn on the full batch of the configurations all three can serve."""
+    wl = W.make(idx, seed=2)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G.set_kernel({"group": B.MOC_KERNEL_GROUP, "warp": B.MOC_KERNEL_WARP, "lane": B.MOC_KERNEL_LANE}[kind])
+    assert_batch_equal(G, O, wl.seqs, wl.lens, B.budget_from_peak(G.no_remat_peak(), 80), f"{kind} {wl.name}")
+    assert B.moc_last_launch_count() >= 1
+
+
+def test_lane_kernel_refuses_what_it_cannot_serve(B):
+    wl = W.make(3, seed=1, B=8)                          # C = 3
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G.set_kernel(B.MOC_KERNEL_LANE)
+    with pytest.raises(B.MocError):
+        G.eval_batch(dev(wl.seqs), dev(wl.lens), BIG)
+    G.set_kernel(B.MOC_KERNEL_AUTO)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    assert_batch_equal(G, O, wl.seqs, wl.lens, BIG, "auto after a refused kind")
+
+
 # ------------------------------------------------------------------ launch shapes, alignment, edges
 @pytest.mark.parametrize("tps,spb", [(0, 0), (0, 4), (0, 8), (0, 12), (0, 16), (32, 1), (32, 8), (32, 16), (64, 4), (128, 2), (256, 1), (256, 3),
                                      (512, 1), (512, 2), (1024, 1)])
