@@ -126,17 +126,18 @@ const char* plan_lane(const moc_graph* g, size_t smem_cap, Plan* out) {
         const LaneLayout& L = g->lane[li];
         if (!L.ok) continue;
         if (forced && g->want_a && g->want_a != gsz) continue;
-        const size_t rec_b = 16 * (size_t)S * L.n_bundles, w_b = align16(8 * (size_t)S * L.n_bundles),
-                     succ_b = align16(4 * (size_t)L.succ_len), word_b = align16(4 * (size_t)gsz * (n + 3)),
+        const size_t rec_b = 32 * (size_t)S * L.n_bundles, succ_b = align16(4 * (size_t)L.succ_len),
+                     part_b = 2 * align16(32 * msz * ((size_t)gsz + 1)),
+                     word_b = moc::lane_special(gsz) + align16((size_t)moc::lane_word_row(gsz) * (n + 1)),
                      delta_b = align16(msz * gsz * (size_t)(t_max + 3));
+        const size_t sm = rec_b + succ_b + part_b + word_b + delta_b;
+        if (sm > smem_cap) continue;
         int best_w = 0, best_nb = 0, best_kp = 0;
         for (int w = 32; w >= 2; w -= 2) {
             if (forced && g->want_b && g->want_b != w) continue;
-            const int Q = w * S;
-            const size_t sm = rec_b + w_b + succ_b + 2 * (size_t)Q * gsz * msz + word_b + delta_b;
-            if (sm > smem_cap) continue;
-            // vectors fetched ahead per sub-lane: enough for a typical row of about 1.3 n steps
-            int kp = (int)(((n * 13 / 10 + 6) / 4 + Q - 1) / Q);
+            // pieces of 128 steps fetched ahead per warp: enough for typical rows of about 1.3 n steps
+            const int64_t blocks = ((n * 13 / 10 + 6) / 4 + 31) / 32;
+            int kp = (int)((blocks * gsz + w - 1) / w);
             kp = std::min(8, std::max(2, (kp + 1) & ~1));
             LaneFn fn = lane_fn(pl.wide, lg, kp);
             if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
@@ -148,17 +149,16 @@ const char* plan_lane(const moc_graph* g, size_t smem_cap, Plan* out) {
             if (warps > best || (warps == best && nb > best_nb && w >= 8)) { best_w = w; best_nb = nb; best_kp = kp; }
         }
         if (best_w == 0) continue;
-        const int Q = best_w * S;
         pl.lane = true;
         pl.lane_fn = lane_fn(pl.wide, lg, best_kp);
         pl.lane_lg = lg;
         pl.G = 32 * best_w / gsz;
         pl.gpc = gsz;
         pl.block = 32 * best_w;
-        pl.smem = rec_b + w_b + succ_b + 2 * (size_t)Q * gsz * msz + word_b + delta_b;
+        pl.smem = sm;
         pl.grid = g->sm_count * best_nb;
         pl.sm_count = g->sm_count;
-        pl.lane_rec_b = (uint32_t)rec_b; pl.lane_w_b = (uint32_t)w_b; pl.lane_succ_b = (uint32_t)succ_b;
+        pl.lane_rec_b = (uint32_t)rec_b; pl.lane_succ_b = (uint32_t)succ_b;
         pl.lane_word_b = (uint32_t)word_b; pl.lane_delta_b = (uint32_t)delta_b;
         pl.valid = true;
         *out = pl;
@@ -306,21 +306,24 @@ int ensure(void** ptr, size_t* cap, size_t need) {
 }
 
 
-// Durations of the sequence-per-lane layouts: w | 1 << 40 (counts the node when it has two copies)
-// | 1 << 52 when the node's cap C_v is 1.
-int upload_lane_w(moc_graph* g) {
+// Words 4-5 of the node records of the sequence-per-lane layouts: w | 1 << 40 (counts the node when
+// it has two copies) | 1 << 52 when the node's cap C_v is 1.  Uploads both record arrays.
+int upload_lane_rec(moc_graph* g) {
     for (int li = 0; li < 3; ++li) {
         LaneLayout& L = g->lane[li];
         if (!L.ok) continue;
-        std::vector<uint64_t> wx(L.h_node.size());
-        for (size_t r = 0; r < wx.size(); ++r) {
+        for (size_t r = 0; r < L.h_node.size(); ++r) {
             const int32_t v = L.h_node[r];
-            if (v < 0) { wx[r] = 0; continue; }
-            uint64_t x = (uint64_t)g->h_w[v] | (uint64_t(1) << moc::kLaneCntShift);
-            if (!g->h_cap.empty() && g->h_cap[v] == 1) x |= uint64_t(1) << moc::kLaneCapShift;
-            wx[r] = x;
+            uint64_t x = 0;
+            if (v >= 0) {
+                x = (uint64_t)g->h_w[v] | (uint64_t(1) << moc::kLaneCntShift);
+                if (!g->h_cap.empty() && g->h_cap[v] == 1) x |= uint64_t(1) << moc::kLaneCapShift;
+            }
+            L.h_rec32[8 * r + 4] = L.h_rec64[8 * r + 4] = (uint32_t)(x & 0xFFFFFFFFu);
+            L.h_rec32[8 * r + 5] = L.h_rec64[8 * r + 5] = (uint32_t)(x >> 32);
         }
-        MOC_CUDA(cudaMemcpy(L.d_w, wx.data(), wx.size() * 8, cudaMemcpyHostToDevice));
+        MOC_CUDA(cudaMemcpy(L.d_rec32, L.h_rec32.data(), L.h_rec32.size() * 4, cudaMemcpyHostToDevice));
+        MOC_CUDA(cudaMemcpy(L.d_rec64, L.h_rec64.data(), L.h_rec64.size() * 4, cudaMemcpyHostToDevice));
     }
     return MOC_OK;
 }
@@ -329,7 +332,6 @@ int upload_lane_w(moc_graph* g) {
 // Nodes in order of falling out-degree (a sink counts one: its made-up successor), S consecutive
 // nodes form a bundle and share a row count; entry (k, h) of a bundle is the byte offset of the
 // word row of the k-th successor of its h-th node, the node's own row once its list is used up.
-// Rows of the word array: 0..n-1 nodes, n spare (ids out of range), n+1 holds T, n+2 holds (1, 1).
 int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, const std::vector<int32_t>& succ,
                        const int64_t* m, const std::vector<int32_t>& m32) {
     const int32_t n = g->n;
@@ -345,9 +347,10 @@ int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, con
         const int32_t nb = (n + S - 1) / S;
         std::vector<int32_t> node((size_t)nb * S, -1);
         for (int32_t i = 0; i < n; ++i) node[i] = order[i];
-        std::vector<uint4> rec32(node.size()), rec64(node.size());
+        std::vector<uint32_t> rec32(node.size() * 8, 0u), rec64(node.size() * 8, 0u);
         std::vector<uint32_t> se;
-        const uint32_t row_b = 4u * (uint32_t)gsz;
+        const uint32_t row_b = moc::lane_word_row(gsz);
+        const uint32_t t_row = 0u - moc::lane_special(gsz), one_row = t_row + row_b;   // relative to the first node row
         for (int32_t bd = 0; bd < nb; ++bd) {
             int rows = 0;
             for (int h = 0; h < S; ++h)
@@ -356,42 +359,41 @@ int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, con
             for (int k = 0; k < rows; ++k)
                 for (int h = 0; h < S; ++h) {
                     const int32_t v = node[(size_t)bd * S + h];
-                    uint32_t row;
-                    if (v < 0) row = (uint32_t)n + 2;
-                    else if (k < succ_start[v + 1] - succ_start[v]) row = (uint32_t)succ[succ_start[v] + k];
-                    else if (k == 0) row = (uint32_t)n + 1;          // a sink: the word that holds T
-                    else row = (uint32_t)v;
-                    se.push_back(row * row_b);
+                    uint32_t off;
+                    if (v < 0) off = one_row;
+                    else if (k < succ_start[v + 1] - succ_start[v]) off = (uint32_t)succ[succ_start[v] + k] * row_b;
+                    else if (k == 0) off = t_row;                    // a sink: the word that holds T
+                    else off = (uint32_t)v * row_b;
+                    se.push_back(off);
                 }
             for (int h = 0; h < S; ++h) {
                 const size_t r = (size_t)bd * S + h;
                 const int32_t v = node[r];
-                const uint32_t x = (v >= 0 ? (uint32_t)v : (uint32_t)n + 2) * row_b;
-                const uint32_t y = (first + (uint32_t)h) | ((uint32_t)rows << 24);
                 const uint64_t mv = v >= 0 ? (uint64_t)m[v] : 0;
-                rec32[r] = make_uint4(x, y, v >= 0 ? (uint32_t)m32[v] : 0u, 0u);
-                rec64[r] = make_uint4(x, y, (uint32_t)(mv & 0xFFFFFFFFu), (uint32_t)(mv >> 32));
+                rec32[8 * r + 0] = rec64[8 * r + 0] = v >= 0 ? (uint32_t)v * row_b : one_row;
+                rec32[8 * r + 1] = rec64[8 * r + 1] = (4u * (first + (uint32_t)h)) | ((uint32_t)rows << 24);
+                rec32[8 * r + 2] = v >= 0 ? (uint32_t)m32[v] : 0u;
+                rec64[8 * r + 2] = (uint32_t)(mv & 0xFFFFFFFFu);
+                rec64[8 * r + 3] = (uint32_t)(mv >> 32);
             }
         }
-        while (se.size() % 4) se.push_back(((uint32_t)n + 2) * row_b);
-        if (se.empty()) se.assign(4, ((uint32_t)n + 2) * row_b);
-        if (se.size() >= (size_t(1) << 24)) continue;
-        cudaError_t e = cudaMalloc(&L.d_rec32, rec32.size() * 16);
-        if (e == cudaSuccess) e = cudaMalloc(&L.d_rec64, rec64.size() * 16);
-        if (e == cudaSuccess) e = cudaMalloc((void**)&L.d_w, align16(node.size() * 8));
+        while (se.size() % 4) se.push_back(one_row);
+        if (se.empty()) se.assign(4, one_row);
+        if (se.size() * 4 + 64 >= (size_t(1) << 24)) continue;
+        cudaError_t e = cudaMalloc(&L.d_rec32, rec32.size() * 4);
+        if (e == cudaSuccess) e = cudaMalloc(&L.d_rec64, rec64.size() * 4);
         if (e == cudaSuccess) e = cudaMalloc((void**)&L.d_succ, se.size() * 4);
-        if (e == cudaSuccess) e = cudaMemcpy(L.d_rec32, rec32.data(), rec32.size() * 16, cudaMemcpyHostToDevice);
-        if (e == cudaSuccess) e = cudaMemcpy(L.d_rec64, rec64.data(), rec64.size() * 16, cudaMemcpyHostToDevice);
-        if (e == cudaSuccess) e = cudaMemset(L.d_w, 0, align16(node.size() * 8));
         if (e == cudaSuccess) e = cudaMemcpy(L.d_succ, se.data(), se.size() * 4, cudaMemcpyHostToDevice);
         if (e != cudaSuccess)
             return fail(e == cudaErrorMemoryAllocation ? MOC_ERR_NOMEM : MOC_ERR_CUDA, "moc_graph_create: %s", cudaGetErrorString(e));
         L.n_bundles = nb;
         L.succ_len = (int64_t)se.size();
         L.h_node = node;
+        L.h_rec32 = rec32;
+        L.h_rec64 = rec64;
         L.ok = true;
     }
-    return upload_lane_w(g);
+    return upload_lane_rec(g);
 }
 
 moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
@@ -465,7 +467,6 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.M = M;
         q.base_dur = g->sum_w;
         q.rec = (const uint4*)(pl.wide ? L.d_rec64 : L.d_rec32);
-        q.wrec = L.d_w;
         q.succ = L.d_succ;
         q.seqs = seqs;
         q.lens = lens;
@@ -473,7 +474,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.out_peak = out_peak;
         q.out_dur = out_dur;
         q.out_status = out_feasible;
-        q.rec_bytes = pl.lane_rec_b; q.w_bytes = pl.lane_w_b; q.succ_bytes = pl.lane_succ_b;
+        q.rec_bytes = pl.lane_rec_b; q.succ_bytes = pl.lane_succ_b;
         q.word_bytes = pl.lane_word_b; q.delta_bytes = pl.lane_delta_b;
         MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.lane_fn, q));
     } else if (pl.pair) {
@@ -846,7 +847,7 @@ int moc_graph_set_node_caps(moc_graph* g, const int32_t* caps) {
     }
     int rc = upload_wslot(g);
     if (rc != MOC_OK) return rc;
-    return upload_lane_w(g);
+    return upload_lane_rec(g);
 }
 
 int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b) {
@@ -919,7 +920,6 @@ void moc_graph_destroy(moc_graph* g) {
     for (int li = 0; li < 3; ++li) {
         cudaFree(g->lane[li].d_rec32);
         cudaFree(g->lane[li].d_rec64);
-        cudaFree(g->lane[li].d_w);
         cudaFree(g->lane[li].d_succ);
     }
     delete g;

@@ -37,7 +37,7 @@ struct Plan {
     bool lane = false;
     LaneFn lane_fn = nullptr;
     int lane_lg = 0;               // log2 of the sequences per group
-    uint32_t lane_rec_b = 0, lane_w_b = 0, lane_succ_b = 0, lane_word_b = 0, lane_delta_b = 0;
+    uint32_t lane_rec_b = 0, lane_succ_b = 0, lane_word_b = 0, lane_delta_b = 0;
 };
 
 // Graph in the order the sequence-per-lane kernel walks it, for one group size (S = 32 / g sub-lanes).
@@ -45,11 +45,11 @@ struct LaneLayout {
     bool ok = false;
     int32_t n_bundles = 0;
     int64_t succ_len = 0;                 // entries of the successor array (a multiple of 4)
-    void* d_rec32 = nullptr;              // uint4 records with 32-bit / 64-bit output sizes
+    void* d_rec32 = nullptr;              // 32-byte records with 32-bit / 64-bit output sizes
     void* d_rec64 = nullptr;
-    uint64_t* d_w = nullptr;
     uint32_t* d_succ = nullptr;
     std::vector<int32_t> h_node;          // node of every slot (-1: none)
+    std::vector<uint32_t> h_rec32, h_rec64;   // host copies of the records (durations and caps are patched in)
 };
 
 
