@@ -404,7 +404,7 @@ int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t seq
  *                     (0 = choose); any C <= MOC_MAX_COPIES.  Same as moc_graph_set_launch(a, b).
  *   MOC_KERNEL_WARP   one warp per sequence, b warps per block (0 or 4..16), a = 0; C <= 2.
  *   MOC_KERNEL_LANE   one sequence per lane: a block keeps a group of a sequences (0, 8, 16, 32)
- *                     on chip and its b warps (0 or an even number 2..32) share the work on them;
+ *                     on chip and its b warps (0, 8, 16, 24 or 32; a multiple of a) share the work on them;
  *                     C <= 2 and a graph whose state for a group fits in shared memory.
  * MOC_ERR_ARG for an unknown kind or shape; a kind that cannot serve the graph with its current C
  * is reported by the next moc_eval_batch (MOC_ERR_ARG), which evaluates nothing.

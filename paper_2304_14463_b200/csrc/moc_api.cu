@@ -133,11 +133,11 @@ const char* plan_lane(const moc_graph* g, size_t smem_cap, Plan* out) {
         const size_t sm = rec_b + succ_b + part_b + word_b + delta_b;
         if (sm > smem_cap) continue;
         int best_w = 0, best_nb = 0, best_kp = 0;
-        for (int w = 32; w >= 2; w -= 2) {
+        for (int w = 32; w >= gsz; w -= gsz) {    // a whole number of warps per row of the group
             if (forced && g->want_b && g->want_b != w) continue;
             // pieces of 128 steps fetched ahead per warp: enough for typical rows of about 1.3 n steps
-            const int64_t blocks = ((n * 13 / 10 + 6) / 4 + 31) / 32;
-            int kp = (int)((blocks * gsz + w - 1) / w);
+            const int64_t pieces = ((n * 13 / 10 + 6) / 4 + 31) / 32;
+            int kp = (int)((pieces * gsz + w - 1) / w);
             kp = std::min(8, std::max(2, (kp + 1) & ~1));
             LaneFn fn = lane_fn(pl.wide, lg, kp);
             if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); continue; }
@@ -183,7 +183,11 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
     const size_t smem_cap = g->smem_optin > 1024 ? g->smem_optin - 1024 : 0;  // 1 KB per block is reserved
     const int kind = profile ? MOC_KERNEL_GROUP : g->want_kind;
     const bool shape_given = g->want_G != 0 || g->want_gpc != 0;       // moc_graph_set_launch
-    if (kind == MOC_KERNEL_LANE || (kind == MOC_KERNEL_AUTO && !shape_given && !profile)) {
+    // Order of preference when nothing is forced: warp per sequence, then sequence per lane (it also
+    // serves graphs whose degrees are too uneven for the warp kernel's padded successor tiles), then
+    // the thread-group kernel, which serves everything.
+    const bool warp_ok = C <= 2 && g->d_rec32 != nullptr;
+    if (kind == MOC_KERNEL_LANE || (kind == MOC_KERNEL_AUTO && !shape_given && !warp_ok)) {
         const char* why = plan_lane(g, smem_cap, &pl);
         if (!why) {
             *out = pl;
@@ -191,7 +195,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         }
         if (kind == MOC_KERNEL_LANE) return fail(MOC_ERR_ARG, "the sequence-per-lane kernel cannot serve this graph: %s", why);
     }
-    if (kind == MOC_KERNEL_WARP && (C > 2 || g->d_rec32 == nullptr))
+    if (kind == MOC_KERNEL_WARP && !warp_ok)
         return fail(MOC_ERR_ARG, "the warp-per-sequence kernel cannot serve this graph (C > 2 or degrees too uneven)");
     if (!profile && g->want_G == 0 && kind != MOC_KERNEL_GROUP && C <= 2 && g->d_rec32 != nullptr) {
         // warp-per-sequence fast path
@@ -373,8 +377,11 @@ int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, con
                 rec32[8 * r + 0] = rec64[8 * r + 0] = v >= 0 ? (uint32_t)v * row_b : one_row;
                 rec32[8 * r + 1] = rec64[8 * r + 1] = (4u * (first + (uint32_t)h)) | ((uint32_t)rows << 24);
                 rec32[8 * r + 2] = v >= 0 ? (uint32_t)m32[v] : 0u;
+                rec32[8 * r + 3] = 0u - rec32[8 * r + 2];
                 rec64[8 * r + 2] = (uint32_t)(mv & 0xFFFFFFFFu);
                 rec64[8 * r + 3] = (uint32_t)(mv >> 32);
+                rec64[8 * r + 6] = (uint32_t)((0 - mv) & 0xFFFFFFFFu);
+                rec64[8 * r + 7] = (uint32_t)((0 - mv) >> 32);
             }
         }
         while (se.size() % 4) se.push_back(one_row);
@@ -861,7 +868,7 @@ int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b) {
                  !(a && b && a * b > 1024);
             break;
         case MOC_KERNEL_WARP: ok = a == 0 && (b == 0 || (b >= 4 && b <= 16)); break;
-        case MOC_KERNEL_LANE: ok = (a == 0 || a == 8 || a == 16 || a == 32) && (b == 0 || (b >= 2 && b <= 32 && b % 2 == 0)); break;
+        case MOC_KERNEL_LANE: ok = (a == 0 || a == 8 || a == 16 || a == 32) && (b == 0 || (b >= 8 && b <= 32 && b % 8 == 0)); break;
         default: break;
     }
     if (!ok) return fail(MOC_ERR_ARG, "moc_graph_set_kernel: unsupported kind or shape (%d, %d, %d)", kind, a, b);

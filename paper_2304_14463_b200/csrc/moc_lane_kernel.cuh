@@ -72,8 +72,8 @@ __host__ __device__ constexpr uint32_t lane_word_row(int g) { return 4u * ((uint
 __host__ __device__ constexpr uint32_t lane_special(int g) { return (2u * lane_word_row(g) + 15u) & ~15u; }
 
 // Node record, 32 bytes: word 0 = byte offset of the node's row from the first node row, word 1 =
-// byte offset of its first successor entry | rows of its bundle << 24, words 2-3 = m (int32: low
-// word only), words 4-5 = w | 1 << 40 | (C_v == 1) << 52.  Entry (k, h) of a bundle sits S * k + h
+// byte offset of its first successor entry | rows of its bundle << 24, words 2-3 = m (int32: word 2
+// = m, word 3 = -m), words 4-5 = w | 1 << 40 | (C_v == 1) << 52, words 6-7 = -m (int64 only).  Entry (k, h) of a bundle sits S * k + h
 // entries after the bundle's first entry and is itself the byte offset of a row; lists shorter than the
 // bundle's rows are padded with the node's own row, which is neutral for both reductions.
 constexpr uint64_t kLaneDurMask = (uint64_t(1) << 40) - 1;   // bits 0..39: sum of w over second copies
@@ -129,6 +129,11 @@ __device__ __forceinline__ void lane_second_copy(uint32_t x, uint32_t y, uint32_
                  : "+r"(acc_lo), "+r"(acc_hi) : "r"(x), "r"(y), "r"(a0), "l"(v0), "r"(a1), "l"(v1), "r"(inc_lo), "r"(inc_hi) : "memory");
 }
 
+// Makes a value opaque to the compiler at this point: it is then kept in its register instead of
+// being recomputed from the kernel parameters wherever it is used (the hot loops are short of
+// instruction slots, not of registers).
+#define MOC_LANE_KEEP(x) asm volatile("" : "+r"(x))
+
 // Vector k of a row covers the steps 4k - a .. 4k - a + 3 (a = ints between the 16-byte boundary
 // below the row and the row).  Steps outside [0, T) come back as -1, which stage 1 sends to the spare row.
 __device__ __forceinline__ int4 lane_load_vec(const int32_t* row, int k, int a, int T) {
@@ -157,22 +162,31 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
     __shared__ unsigned long long s_acc[g];
 
     const int lane = threadIdx.x & 31, j = lane & (g - 1), h = lane >> LG;
-    const int W = blockDim.x >> 5;
+    int W = blockDim.x >> 5;
+    MOC_LANE_KEEP(W);
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
     const int Q = W * S, q = warp * S + h;
     const int QS = min(Q, 32);                 // chunks of the prefix sum (one warp puts them together)
-    const int n = p.n, n_bundles = p.n_bundles;
+    int n = p.n, n_bundles = p.n_bundles;
+    MOC_LANE_KEEP(n);
+    MOC_LANE_KEEP(n_bundles);
 
     // ---- shared-memory map: graph | chunk sums | chunk maxima | special rows, words | deltas
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
-    const uint32_t a_rec = sbase, a_succ = a_rec + p.rec_bytes;
+    const uint32_t a_rec = sbase;
+    uint32_t a_succ = a_rec + p.rec_bytes;
     const uint32_t part_bytes = (32u * kPartRow + 15u) & ~15u;
     const uint32_t a_run = a_succ + p.succ_bytes, a_top = a_run + part_bytes;
-    const uint32_t a_word = a_top + part_bytes + kSpecial;                    // first node row
+    uint32_t a_word = a_top + part_bytes + kSpecial;                          // first node row
     const uint32_t a_delta = a_word - kSpecial + p.word_bytes;
-    const uint32_t wlane = a_word + 4u * j;                                   // word of sequence j in the first node row
-    const uint32_t dlane = a_delta + kMemRow + (uint32_t)sizeof(MemT) * j;    // delta of sequence j at step 0
-    const uint32_t dlane1 = dlane - kMemRow;                                  // ... at step -1
+    uint32_t wlane = a_word + 4u * j;                                         // word of sequence j in the first node row
+    uint32_t dlane = a_delta + kMemRow + (uint32_t)sizeof(MemT) * j;          // delta of sequence j at step 0
+    uint32_t dlane1 = dlane - kMemRow;                                        // ... at step -1
+    MOC_LANE_KEEP(a_succ);
+    MOC_LANE_KEEP(a_word);
+    MOC_LANE_KEEP(wlane);
+    MOC_LANE_KEEP(dlane);
+    MOC_LANE_KEEP(dlane1);
 
     // ---- this block's groups: [grp, grp_end) of ceil(B / g); sum of the lengths in front of them
     const int n_groups = (p.B + g - 1) >> LG;
@@ -245,18 +259,21 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
             s_T[gi & 1][j] = (len >= n && len <= p.max_T) ? len : 0;
         }
     };
-    // Stage 1 works in pieces: piece u is the part of row u % g that the vectors 32 (u / g) .. + 31
-    // cover, lane l its vector 32 (u / g) + l; a warp takes the pieces warp, warp + W, ...  The first
-    // KP pieces of a warp are requested one group ahead so that they arrive behind other work.
+    // Stage 1 works in pieces of 32 vectors (128 steps).  The block has a whole number of warps per
+    // row: this warp takes row rj and of its pieces number pk0, pk0 + pstep, ...; lane l takes vector l
+    // of a piece.  The warp's first KP pieces are requested one group ahead so that they arrive behind
+    // other work.
+    const int rj = warp & (g - 1), pk0 = warp >> LG, pstep = W >> LG;
     int4 pre[KP];
     auto prefetch_group = [&](int gi) {
+        const int32_t Tj = s_T[gi & 1][rj];
+        const int32_t* row = p.seqs + s_off[gi & 1][rj];
+        const int a = (int)((reinterpret_cast<uintptr_t>(row) >> 2) & 3);
+        const int nvec = Tj ? (Tj + a + 3) >> 2 : 0;
 #pragma unroll
         for (int i = 0; i < KP; ++i) {
-            const int u = warp + i * W, jj = u & (g - 1), k = ((u >> LG) << 5) + lane;
-            const int32_t T = s_T[gi & 1][jj];
-            const int32_t* row = p.seqs + s_off[gi & 1][jj];
-            const int a = (int)((reinterpret_cast<uintptr_t>(row) >> 2) & 3);
-            if (T != 0 && k < ((T + a + 3) >> 2)) pre[i] = lane_load_vec(row, k, a, T);
+            const int k = ((pk0 + i * pstep) << 5) + lane;
+            if (k < nvec) pre[i] = lane_load_vec(row, k, a, Tj);
         }
     };
     if (grp < grp_end) {
@@ -269,12 +286,15 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
     for (; grp < grp_end; ++grp) {
         const int buf = grp & 1;
         const int32_t T = s_T[buf][j];      // 0: nothing to evaluate in this lane
-        const int Tmax = __reduce_max_sync(0xFFFFFFFFu, T);
         // ---- stage 1: occurrence words
         {
-            const int n_pieces = ((((Tmax + 6) >> 2) + 31) >> 5) << LG;
-            auto put4 = [&](const int4 v, const uint32_t wj, const int t1) {
-                uint32_t val = (uint32_t)t1 * 0x10001u;
+            const int32_t Tj = s_T[buf][rj];
+            const int32_t* row = p.seqs + s_off[buf][rj];
+            const int a = (int)((reinterpret_cast<uintptr_t>(row) >> 2) & 3);
+            const int nvec = Tj ? (Tj + a + 3) >> 2 : 0;
+            const uint32_t wj = a_word + 4u * (uint32_t)rj;
+            auto put4 = [&](const int4 v, const int k) {
+                uint32_t val = (uint32_t)(4 * k - a + 1) * 0x10001u;
                 const int32_t id[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -286,18 +306,10 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
             };
 #pragma unroll
             for (int i = 0; i < KP; ++i) {
-                const int u = warp + i * W, jj = u & (g - 1), k = ((u >> LG) << 5) + lane;
-                const int32_t Tj = s_T[buf][jj];
-                const int a = (int)(((reinterpret_cast<uintptr_t>(p.seqs) >> 2) + (uint64_t)s_off[buf][jj]) & 3);
-                if (u < n_pieces && Tj != 0 && k < ((Tj + a + 3) >> 2)) put4(pre[i], a_word + 4u * jj, 4 * k - a + 1);
+                const int k = ((pk0 + i * pstep) << 5) + lane;
+                if (k < nvec) put4(pre[i], k);
             }
-            for (int u = warp + KP * W; u < n_pieces; u += W) {
-                const int jj = u & (g - 1), k = ((u >> LG) << 5) + lane;
-                const int32_t Tj = s_T[buf][jj];
-                const int32_t* row = p.seqs + s_off[buf][jj];
-                const int a = (int)((reinterpret_cast<uintptr_t>(row) >> 2) & 3);
-                if (Tj != 0 && k < ((Tj + a + 3) >> 2)) put4(lane_load_vec(row, k, a, Tj), a_word + 4u * jj, 4 * k - a + 1);
-            }
+            for (int k = ((pk0 + KP * pstep) << 5) + lane; k < nvec; k += pstep << 5) put4(lane_load_vec(row, k, a, Tj), k);
         }
         __syncthreads();
 
@@ -306,10 +318,12 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
         {
             uint32_t vmin = 0xFFFFFFFFu, depw = 0, acc_lo = 0, acc_hi = 0;
             uint32_t prec = a_rec + 32u * (uint32_t)q;
-            const uint32_t rec_step = 32u * (uint32_t)Q;
-            for (int bd = warp; bd < n_bundles; bd += W, prec += rec_step) {
+            uint32_t rec_step = 32u * (uint32_t)Q, rec_end = a_rec + 32u * (uint32_t)(n_bundles * S);
+            MOC_LANE_KEEP(rec_step);
+            MOC_LANE_KEEP(rec_end);
+            for (; prec < rec_end; prec += rec_step) {
                 const uint4 rec = lds_v4(prec);
-                const uint2 wx = lds_v2(prec + 16);
+                const uint4 rec2 = lds_v4(prec + 16);      // w and flags; -m of 64 bits
                 const uint32_t own = lds_u32(wlane + rec.x);
                 const uint32_t sw = swap_halves(own);
                 const uint32_t mn = min_u16x2(own, sw), mx = max_u16x2(own, sw);   // (a, a), (b, b)
@@ -330,13 +344,18 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
                 const uint32_t gg = max_u16x2(__byte_perm(Ga, Gb, 0x5410), __byte_perm(Ga, Gb, 0x7632));  // (best Ga, best Gb)
                 const uint32_t ab = __byte_perm(mn, mx, 0x7610);                   // (a, b)
                 const uint32_t v = gg + ab;                                        // (end of b, end of a) mod 2^16
-                MemT m;
-                if constexpr (sizeof(MemT) == 4) m = (MemT)rec.z;
-                else m = (MemT)((uint64_t)rec.z | ((uint64_t)rec.w << 32));
+                MemT m, neg_m;
+                if constexpr (sizeof(MemT) == 4) {
+                    m = (MemT)rec.z;
+                    neg_m = (MemT)rec.w;
+                } else {
+                    m = (MemT)((uint64_t)rec.z | ((uint64_t)rec.w << 32));
+                    neg_m = (MemT)((uint64_t)rec2.z | ((uint64_t)rec2.w << 32));
+                }
                 red_add_shared(dlane1 + (ab >> 16) * kMemRow, m);
-                red_add_shared(dlane + (v & 0xFFFFu) * kMemRow, (MemT)(-m));
-                lane_second_copy(mn, mx, dlane1 + (ab & 0xFFFFu) * kMemRow, m, dlane + (v >> 16) * kMemRow, (MemT)(-m),
-                                 acc_lo, acc_hi, wx.x, wx.y);
+                red_add_shared(dlane + (v & 0xFFFFu) * kMemRow, neg_m);
+                lane_second_copy(mn, mx, dlane1 + (ab & 0xFFFFu) * kMemRow, m, dlane + (v >> 16) * kMemRow, neg_m,
+                                 acc_lo, acc_hi, rec2.x, rec2.y);
                 vmin = min(vmin, own);
             }
             atomicMin(&s_vmin[j], vmin);
@@ -350,7 +369,7 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
         const bool more = grp + 1 < grp_end;
         if (more) prefetch_group(grp + 1);
         {
-            const int E = Tmax + 2;                       // steps 0 .. Tmax + 1 can hold something
+            const int E = __reduce_max_sync(0xFFFFFFFFu, T) + 2;      // steps 0 .. Tmax + 1 can hold something
             const int L = (E + QS - 1) / QS;
             if (q < QS) {
                 const int t0 = q * L, t1 = min(t0 + L, E);
