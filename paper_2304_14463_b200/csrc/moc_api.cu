@@ -186,7 +186,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
     // Order of preference when nothing is forced: warp per sequence, then sequence per lane (it also
     // serves graphs whose degrees are too uneven for the warp kernel's padded successor tiles), then
     // the thread-group kernel, which serves everything.
-    const bool warp_ok = C <= 2 && g->d_rec32 != nullptr;
+    const bool warp_ok = C <= 2 && g->d_rec32 != nullptr && (__int128)C * g->sum_w < ((__int128)1 << 48);
     if (kind == MOC_KERNEL_LANE || (kind == MOC_KERNEL_AUTO && !shape_given && !warp_ok)) {
         const char* why = plan_lane(g, smem_cap, &pl);
         if (!why) {
@@ -196,17 +196,16 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
         if (kind == MOC_KERNEL_LANE) return fail(MOC_ERR_ARG, "the sequence-per-lane kernel cannot serve this graph: %s", why);
     }
     if (kind == MOC_KERNEL_WARP && !warp_ok)
-        return fail(MOC_ERR_ARG, "the warp-per-sequence kernel cannot serve this graph (C > 2 or degrees too uneven)");
-    if (!profile && g->want_G == 0 && kind != MOC_KERNEL_GROUP && C <= 2 && g->d_rec32 != nullptr) {
+        return fail(MOC_ERR_ARG, "the warp-per-sequence kernel cannot serve this graph (C > 2, degrees too uneven or C * sum(w) >= 2^48)");
+    if (!profile && g->want_G == 0 && kind != MOC_KERNEL_GROUP && warp_ok) {
         // warp-per-sequence fast path
         const size_t msz = pl.wide ? 8 : 4, per_vec = 16 / msz;
-        const size_t nvec_d = (t_max + 1 + per_vec - 1) / per_vec;
+        const size_t nvec_d = (t_max + 2 + per_vec - 1) / per_vec;
         const size_t v_max = ((nvec_d + 31) / 32) | 1;
-        const size_t rec_b = (pl.wide ? sizeof(moc::NodeRec<int64_t>) : sizeof(moc::NodeRec<int32_t>)) * 64 * (size_t)g->n_tiles,
-                     col_b = align16(4 * (size_t)g->n_tiles), jds_b = align16(4 * (size_t)g->sell_len),
+        const size_t rec_b = (pl.wide ? 16 : 8) * 64 * (size_t)g->n_tiles, jds_b = align16(4 * (size_t)g->sell_len),
                      word_b = align16(4 * (n + 2)), delta_b = moc::kPairDeltaFront + 32 * v_max * 16;
         const size_t w_b = 8 * 64 * (size_t)g->n_tiles;
-        const size_t graph_b = rec_b + w_b + col_b + jds_b, warp_b = word_b + moc::kPairWordTail + delta_b;
+        const size_t graph_b = rec_b + w_b + jds_b, warp_b = word_b + moc::kPairWordTail + delta_b;
         // vectors of the next row fetched ahead per lane: enough for a typical row of about 1.3 n steps
         const int pre = n < 256 ? 0 : (int)std::min<int64_t>(5, (n * 13 / 10 + 96) / 128);
         PairFn fn = pair_fn(pl.wide, pre);
@@ -232,7 +231,7 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             pl.block = 32 * best_wpb;
             pl.smem = graph_b + best_wpb * warp_b;
             pl.grid = g->sm_count * best_nb;
-            pl.rec_bytes = (uint32_t)rec_b; pl.w_bytes = (uint32_t)w_b; pl.tile_bytes = (uint32_t)col_b;
+            pl.rec_bytes = (uint32_t)rec_b; pl.w_bytes = (uint32_t)w_b;
             pl.sell_bytes = (uint32_t)jds_b; pl.word_bytes = (uint32_t)word_b; pl.delta_bytes = (uint32_t)delta_b;
             cudaError_t e = raise_smem_limit((const void*)fn, g->smem_optin);
             if (e != cudaSuccess) return fail(MOC_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
@@ -487,14 +486,11 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
     } else if (pl.pair) {
         moc::PairParams q{};
         q.n = g->n;
-        q.sell_len = g->sell_len;
         q.n_tiles = g->n_tiles;
-        q.sum_bias = (uint32_t)(64 * g->n_tiles - g->n);
         q.max_T = g->C * g->n;
         q.rec = pl.wide ? g->d_rec64 : g->d_rec32;
-        q.wslot = g->d_wslot;
+        q.wslot = (const uint64_t*)g->d_wslot;
         q.sell = g->d_sell;
-        q.tile = g->d_tile;
         q.base_dur = g->sum_w;
         q.seqs = seqs;
         q.lens = lens;
@@ -504,7 +500,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.out_peak = out_peak;
         q.out_dur = out_dur;
         q.out_status = out_feasible;
-        q.rec_bytes = pl.rec_bytes; q.w_bytes = pl.w_bytes; q.tile_bytes = pl.tile_bytes; q.sell_bytes = pl.sell_bytes;
+        q.rec_bytes = pl.rec_bytes; q.w_bytes = pl.w_bytes; q.sell_bytes = pl.sell_bytes;
         q.word_bytes = pl.word_bytes; q.delta_bytes = pl.delta_bytes;
         MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.pair_fn, q));
     } else {
@@ -569,6 +565,8 @@ int eval_rows(const moc_graph* g, const int64_t* offs, const int32_t* seqs, cons
 }  // namespace moc_host
 
 extern "C" {
+
+static int upload_wslot(moc_graph* g);
 
 const char* moc_last_error(void) { return g_err; }
 int moc_last_launch_count(void) { return g_launches; }
@@ -655,7 +653,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     auto up = [&](void** dst, const void* src, size_t bytes) {
         if (e != cudaSuccess) return;
         e = cudaMalloc(dst, std::max<size_t>(bytes, 16));
-        if (e == cudaSuccess && bytes) e = cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && bytes && src) e = cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice);
     };
     up((void**)&g->d_succ_start, succ_start.data(), ((size_t)n + 1) * 4);
     up((void**)&g->d_succ, succ.data(), (size_t)ne * 4);
@@ -711,28 +709,26 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
             }
             int32_t max_rows = 0;
             for (int32_t d = 0; d < n_tiles; ++d) max_rows = std::max(max_rows, rows[d]);
-            if (sell_len <= 2 * ne + 4096 && sell_len < (1 << 20) && max_rows < (1 << 12)) {
-                const uint32_t word_b = (uint32_t)align16(4 * ((size_t)n + 2));
-                const uint32_t dummy = 4u * (uint32_t)n;
-                std::vector<uint32_t> tile((size_t)n_tiles);
-                std::vector<moc::NodeRec<int32_t>> rec32((size_t)n_halves * 32);
-                std::vector<moc::NodeRec<int64_t>> rec64((size_t)n_halves * 32);
-                std::vector<int64_t> wslot((size_t)n_halves * 32);
-                std::vector<uint32_t> sell((size_t)std::max<int64_t>(sell_len, 1), dummy | (dummy << 16));
+            if (sell_len <= 2 * ne + 4096 && sell_len < (1 << 20) && max_rows < (1 << 12) && 4 * ((int64_t)n + 3) < 65536) {
+                const uint32_t word_b = (uint32_t)align16(4 * ((size_t)n + 2));   // the constant word (1, 1) sits right after the words
+                std::vector<uint32_t> rec32((size_t)n_halves * 32 * 2), rec64((size_t)n_halves * 32 * 4, 0u);
+                // entry (row k, lane l) of a tile: word of the k-th successor of the node in half 0 | same for half 1 << 16;
+                // a list that is used up continues with the node's own word
+                std::vector<uint32_t> sell((size_t)std::max<int64_t>(sell_len, 1), word_b | (word_b << 16));
+                auto own_word = [&](int32_t v) { return v >= 0 ? 4u * (uint32_t)v : word_b; };
                 for (size_t r = 0; r < slot.size(); ++r) {
                     const int32_t v = slot[r];
-                    const uint32_t nd = v >= 0 ? 4u * (uint32_t)v : word_b;
-                    rec32[r].nd = nd;
-                    rec32[r].m = v >= 0 ? m32[v] : 0;
-                    wslot[r] = v >= 0 ? w[v] : 0;
-                    rec64[r].nd = nd;
-                    rec64[r].pad = 0;
-                    rec64[r].m = v >= 0 ? m[v] : 0;
+                    const uint32_t x = own_word(v) | ((uint32_t)rows[r / 64] << 16);
+                    const uint64_t mv = v >= 0 ? (uint64_t)m[v] : 0;
+                    rec32[2 * r + 0] = x;
+                    rec32[2 * r + 1] = v >= 0 ? (uint32_t)m32[v] : 0u;
+                    rec64[4 * r + 0] = x;
+                    rec64[4 * r + 2] = (uint32_t)(mv & 0xFFFFFFFFu);
+                    rec64[4 * r + 3] = (uint32_t)(mv >> 32);
                 }
                 uint32_t pos = 0;
                 std::vector<std::vector<int32_t>> rem(32);
                 for (int32_t d = 0; d < n_tiles; ++d) {
-                    tile[d] = pos | ((uint32_t)rows[d] << 20);
                     for (int32_t h = 0; h < 2; ++h) {
                         std::vector<int32_t> lanes;
                         for (int32_t l = 0; l < 32; ++l) {
@@ -741,24 +737,30 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                             if (v >= 0) rem[l].assign(succ.begin() + succ_start[v], succ.begin() + succ_start[v + 1]);
                             if (v >= 0 && rem[l].empty()) rem[l].push_back(n + 1);  // sink: the word that holds T
                             lanes.push_back(l);
+                            for (int32_t k = 0; k < rows[d]; ++k) {
+                                uint32_t& e = sell[(size_t)pos + 32 * (size_t)k + l];
+                                e = h == 0 ? ((e & 0xFFFF0000u) | own_word(v)) : ((e & 0x0000FFFFu) | (own_word(v) << 16));
+                            }
                         }
                         for (int32_t k = 0; k < rows[d]; ++k) {
                             int used[32] = {0};
+                            for (int32_t l = 0; l < 32; ++l)
+                                if (rem[l].empty()) used[l]++;   // reads its own word, which lies in bank l
                             std::stable_sort(lanes.begin(), lanes.end(),
                                              [&](int32_t x, int32_t y) { return rem[x].size() > rem[y].size(); });
                             for (int32_t l : lanes) {
-                                if (rem[l].empty()) continue;  // stays the dummy
+                                if (rem[l].empty()) continue;  // stays the own word
                                 const bool forced = (int32_t)rem[l].size() >= rows[d] - k;
                                 int pick = -1;
                                 for (size_t c = 0; c < rem[l].size(); ++c)
                                     if (!used[rem[l][c] & 31]) { pick = (int)c; break; }
                                 if (pick < 0 && !forced) continue;  // wait for a row where its bank is free
                                 if (pick < 0) pick = 0;
-                                const uint32_t off = 4u * (uint32_t)rem[l][pick];
                                 used[rem[l][pick] & 31]++;
-                                rem[l].erase(rem[l].begin() + pick);
-                                uint32_t& e = sell[pos + 32 * (uint32_t)k + l];
+                                uint32_t& e = sell[(size_t)pos + 32 * (size_t)k + l];
+                                const uint32_t off = 4u * (uint32_t)rem[l][pick];
                                 e = h == 0 ? ((e & 0xFFFF0000u) | off) : ((e & 0x0000FFFFu) | (off << 16));
+                                rem[l].erase(rem[l].begin() + pick);
                             }
                         }
                     }
@@ -767,11 +769,10 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
                 g->sell_len = (int32_t)sell_len;
                 g->h_slot = slot;
                 g->n_tiles = n_tiles;
-                up(&g->d_rec32, rec32.data(), rec32.size() * sizeof(rec32[0]));
-                up(&g->d_rec64, rec64.data(), rec64.size() * sizeof(rec64[0]));
-                up((void**)&g->d_wslot, wslot.data(), wslot.size() * 8);
-                up((void**)&g->d_sell, sell.data(), (size_t)sell_len * 4);
-                up((void**)&g->d_tile, tile.data(), (size_t)n_tiles * 4);
+                up(&g->d_rec32, rec32.data(), rec32.size() * 4);
+                up(&g->d_rec64, rec64.data(), rec64.size() * 4);
+                up((void**)&g->d_wslot, nullptr, slot.size() * 8);
+                up((void**)&g->d_sell, sell.data(), sell.size() * 4);
             }
         } catch (const std::bad_alloc&) {
             moc_graph_destroy(g);
@@ -787,6 +788,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     }
     try {
         rc = build_lane_layouts(g, succ_start, succ, m, m32);
+        if (rc == MOC_OK) rc = upload_wslot(g);
     } catch (const std::bad_alloc&) {
         rc = fail(MOC_ERR_NOMEM, "host allocation failed");
     }
@@ -812,14 +814,18 @@ int moc_graph_set_max_copies(moc_graph* g, int32_t C) {
     return MOC_OK;
 }
 
-// Uploads the slot durations of the warp-per-sequence layout, with bit 63 marking nodes whose cap is 1.
+// Uploads the slot durations of the warp-per-sequence layout: w | 1 << 48 (counts the node when it has
+// two copies) | 1 << 63 for nodes whose cap C_v is 1.
 static int upload_wslot(moc_graph* g) {
     if (!g->d_wslot) return MOC_OK;
-    std::vector<int64_t> wslot(g->h_slot.size());
+    std::vector<uint64_t> wslot(g->h_slot.size());
     for (size_t r = 0; r < wslot.size(); ++r) {
         const int32_t v = g->h_slot[r];
-        int64_t x = v >= 0 ? g->h_w[v] : 0;
-        if (v >= 0 && !g->h_cap.empty() && g->h_cap[v] == 1) x |= INT64_MIN;
+        uint64_t x = 0;
+        if (v >= 0) {
+            x = (uint64_t)g->h_w[v] | (uint64_t(1) << moc::kPairCntShift);
+            if (!g->h_cap.empty() && g->h_cap[v] == 1) x |= uint64_t(1) << 63;
+        }
         wslot[r] = x;
     }
     MOC_CUDA(cudaMemcpy(g->d_wslot, wslot.data(), wslot.size() * 8, cudaMemcpyHostToDevice));
@@ -918,7 +924,6 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_wslot);
     cudaFree(g->d_cap);
     cudaFree(g->d_sell);
-    cudaFree(g->d_tile);
     cudaFree(g->d_offs);
     cudaFree(g->d_state);
     cudaFree(g->d_stage_seqs);

@@ -28,7 +28,7 @@ struct Plan {
     // fast path for C <= 2: a warp per sequence, graph staged in shared memory
     bool pair = false;
     PairFn pair_fn = nullptr;
-    uint32_t rec_bytes = 0, w_bytes = 0, tile_bytes = 0, sell_bytes = 0, word_bytes = 0;
+    uint32_t rec_bytes = 0, w_bytes = 0, sell_bytes = 0, word_bytes = 0;
     // blocks per SM the fast path reaches with 1..16 warps per block (0: does not fit), and its sizes
     int pair_nb[17] = {0};
     size_t pair_graph_b = 0, pair_warp_b = 0;
@@ -108,13 +108,12 @@ struct moc_graph {
     int32_t sell_len = 0, n_tiles = 0;
     void* d_rec32 = nullptr;  // node records with 32-bit / 64-bit output sizes
     void* d_rec64 = nullptr;
-    int64_t* d_wslot = nullptr;
+    uint64_t* d_wslot = nullptr;
     int32_t* d_cap = nullptr;             // per-node caps C_v, or null: uniform C
     std::vector<int32_t> h_slot;          // node of every slot of the warp-per-sequence layout (-1: none)
     std::vector<int64_t> h_w;             // durations (host copy, to rebuild d_wslot)
     std::vector<int32_t> h_cap;           // per-node caps (empty: uniform)
     uint32_t* d_sell = nullptr;
-    uint32_t* d_tile = nullptr;
     // grow-only scratch; mutable because evaluation takes a const handle
     mutable moc_host::Plan plan_eval, plan_profile;
     mutable int64_t* d_offs = nullptr;

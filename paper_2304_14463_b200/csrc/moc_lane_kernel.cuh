@@ -80,41 +80,6 @@ constexpr uint64_t kLaneDurMask = (uint64_t(1) << 40) - 1;   // bits 0..39: sum 
 constexpr int kLaneCntShift = 40;                             // bits 40..51: number of nodes with two copies
 constexpr int kLaneCapShift = 52;                             // bits 52..63: of those, nodes with C_v = 1
 
-__device__ __forceinline__ uint32_t lds_u32_nv(uint32_t addr) {
-    uint32_t v;
-    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint64_t lds_u64(uint32_t addr) {
-    uint64_t v;
-    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ int32_t lds_mem(uint32_t addr, int32_t) { return (int32_t)lds_u32(addr); }
-__device__ __forceinline__ int64_t lds_mem(uint32_t addr, int64_t) { return (int64_t)lds_u64(addr); }
-__device__ __forceinline__ void sts_mem(uint32_t addr, int32_t v) { sts_u32(addr, (uint32_t)v); }
-__device__ __forceinline__ void sts_mem(uint32_t addr, int64_t v) {
-    asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
-}
-
-__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
-    return v;
-}
-// st.shared.u16 [addr], v  if old != 0
-__device__ __forceinline__ void sts_u16_if_nonzero(uint32_t old, uint32_t addr, uint32_t v) {
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %0, 0;\n\t@q st.shared.u16 [%1], %2;\n\t}" ::"r"(old), "r"(addr),
-                 "h"((uint16_t)v) : "memory");
-}
 // if (x != y): red.shared.add [a0], v0; red.shared.add [a1], v1; acc += inc
 __device__ __forceinline__ void lane_second_copy(uint32_t x, uint32_t y, uint32_t a0, int32_t v0, uint32_t a1, int32_t v1,
                                                  uint32_t& acc_lo, uint32_t& acc_hi, uint32_t inc_lo, uint32_t inc_hi) {
@@ -128,11 +93,6 @@ __device__ __forceinline__ void lane_second_copy(uint32_t x, uint32_t y, uint32_
                  "@q add.cc.u32 %0, %0, %8;\n\t@q addc.u32 %1, %1, %9;\n\t}"
                  : "+r"(acc_lo), "+r"(acc_hi) : "r"(x), "r"(y), "r"(a0), "l"(v0), "r"(a1), "l"(v1), "r"(inc_lo), "r"(inc_hi) : "memory");
 }
-
-// Makes a value opaque to the compiler at this point: it is then kept in its register instead of
-// being recomputed from the kernel parameters wherever it is used (the hot loops are short of
-// instruction slots, not of registers).
-#define MOC_LANE_KEEP(x) asm volatile("" : "+r"(x))
 
 // Vector k of a row covers the steps 4k - a .. 4k - a + 3 (a = ints between the 16-byte boundary
 // below the row and the row).  Steps outside [0, T) come back as -1, which stage 1 sends to the spare row.
@@ -163,13 +123,13 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
 
     const int lane = threadIdx.x & 31, j = lane & (g - 1), h = lane >> LG;
     int W = blockDim.x >> 5;
-    MOC_LANE_KEEP(W);
+    MOC_KEEP(W);
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
     const int Q = W * S, q = warp * S + h;
     const int QS = min(Q, 32);                 // chunks of the prefix sum (one warp puts them together)
     int n = p.n, n_bundles = p.n_bundles;
-    MOC_LANE_KEEP(n);
-    MOC_LANE_KEEP(n_bundles);
+    MOC_KEEP(n);
+    MOC_KEEP(n_bundles);
 
     // ---- shared-memory map: graph | chunk sums | chunk maxima | special rows, words | deltas
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
@@ -182,11 +142,11 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
     uint32_t wlane = a_word + 4u * j;                                         // word of sequence j in the first node row
     uint32_t dlane = a_delta + kMemRow + (uint32_t)sizeof(MemT) * j;          // delta of sequence j at step 0
     uint32_t dlane1 = dlane - kMemRow;                                        // ... at step -1
-    MOC_LANE_KEEP(a_succ);
-    MOC_LANE_KEEP(a_word);
-    MOC_LANE_KEEP(wlane);
-    MOC_LANE_KEEP(dlane);
-    MOC_LANE_KEEP(dlane1);
+    MOC_KEEP(a_succ);
+    MOC_KEEP(a_word);
+    MOC_KEEP(wlane);
+    MOC_KEEP(dlane);
+    MOC_KEEP(dlane1);
 
     // ---- this block's groups: [grp, grp_end) of ceil(B / g); sum of the lengths in front of them
     const int n_groups = (p.B + g - 1) >> LG;
@@ -319,8 +279,8 @@ __global__ void __launch_bounds__(1024, 1) eval_lane_kernel(const LaneParams p) 
             uint32_t vmin = 0xFFFFFFFFu, depw = 0, acc_lo = 0, acc_hi = 0;
             uint32_t prec = a_rec + 32u * (uint32_t)q;
             uint32_t rec_step = 32u * (uint32_t)Q, rec_end = a_rec + 32u * (uint32_t)(n_bundles * S);
-            MOC_LANE_KEEP(rec_step);
-            MOC_LANE_KEEP(rec_end);
+            MOC_KEEP(rec_step);
+            MOC_KEEP(rec_end);
             for (; prec < rec_end; prec += rec_step) {
                 const uint4 rec = lds_v4(prec);
                 const uint4 rec2 = lds_v4(prec + 16);      // w and flags; -m of 64 bits
