@@ -165,7 +165,7 @@ def run_search(args):
     base = workloads.make(WORKLOAD_IDX, seed=1, B=P)
     G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
     P0 = G.no_remat_peak()
-    M = binding.budget_from_peak(P0, PCT)
+    M = workloads.budget_from_peak(P0, PCT)
     d_seqs, d_lens = torch.from_numpy(base.seqs).cuda(), torch.from_numpy(base.lens).cuda()
     S = binding.Search(G, d_seqs, d_lens, M, seed=1)
     if args.incremental or args.samples > 1:
@@ -255,7 +255,7 @@ def run_intervals(args):
     base = workloads.make(WORKLOAD_IDX, seed=1, B=distinct)
     n, C = base.n, base.C
     G = binding.Graph(n, base.edges, base.w, base.m, C)
-    M = binding.budget_from_peak(G.no_remat_peak(), PCT)
+    M = workloads.budget_from_peak(G.no_remat_peak(), PCT)
     # interval form of `distinct` valid sequences: starts = steps, ends = the free steps the library's
     # own profile entry point reports; unused slots parked on the events after the last step
     offs = np.concatenate([[0], np.cumsum(base.lens)])
@@ -352,7 +352,7 @@ def run_edits(args):
     base = workloads.make(WORKLOAD_IDX, seed=1)
     P, per_parent = base.B, 16
     G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
-    M = binding.budget_from_peak(G.no_remat_peak(), PCT)
+    M = workloads.budget_from_peak(G.no_remat_peak(), PCT)
     cache = binding.EditCache(G, P)
     d_seqs, d_lens = torch.from_numpy(base.seqs).cuda(), torch.from_numpy(base.lens).cuda()
     stream = torch.cuda.current_stream()
@@ -505,7 +505,7 @@ def main():
 
     base, ring_host = make_ring(workloads, args.ring, rank, args.workload)
     G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
-    M = binding.budget_from_peak(G.no_remat_peak(), PCT)
+    M = workloads.budget_from_peak(G.no_remat_peak(), PCT)
     ring = []
     for seqs, lens in ring_host:
         B = len(lens)

@@ -111,6 +111,9 @@ int moc_graph_info(const moc_graph* g, int32_t* n, int64_t* n_edges, int32_t* C,
  *                 are valid once the stream has been synchronised.
  * Errors: MOC_ERR_ARG (null pointer with B > 0, B < 0), MOC_ERR_CUDA, MOC_ERR_NOMEM (scratch
  * growth; happens only when B exceeds every earlier B on this handle).
+ * The library cannot see how large a device buffer is: outputs shorter than B entries, or a seqs
+ * buffer shorter than the lengths add up to, make the kernels read or write outside them.  The
+ * caller (the Python binding does it for the outputs) checks the sizes.
  */
 int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens, int32_t B,
                    int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible,
@@ -231,8 +234,10 @@ int moc_check_intervals(const moc_graph* g, const int32_t* s, const int32_t* e, 
  * cache.  The results are exactly those moc_eval_batch gives for the edited sequences.
  *
  * Limits: handles with C <= 2 (the setting of Section 4.3) and C*n <= 65534; per-node caps are honoured.
- * The cache refers to the graph handle (which must outlive it, with unchanged C and caps) and owns
- * about 12 + 12*sizeof(sum type) bytes per step and parent of device memory, allocated by
+ * The cache refers to the graph handle, which must outlive it.  A call of moc_graph_set_max_copies or
+ * moc_graph_set_node_caps makes the cached parents stale: moc_eval_edits (and a moc_search_run that scores
+ * its proposals from a cache) then fails with MOC_ERR_ARG until moc_cache_build has run again; a changed
+ * C needs a new cache.  The cache owns about 12 + 12*sizeof(sum type) bytes per step and parent of device memory, allocated by
  * moc_cache_create only.
  */
 typedef struct moc_cache moc_cache; /* opaque */

@@ -130,12 +130,6 @@ def _host(a, dtype, name):
     return ctypes.c_void_p(a.ctypes.data)
 
 
-def budget_from_peak(peak: int, pct: int) -> int:
-    """M = floor(peak * pct / 100): a budget given as a percentage of a no-rematerialization peak
-    (Section 4.3; the budgets printed there equal this rounding of a common integer peak)."""
-    return int(peak) * int(pct) // 100
-
-
 def moc_graph_create(n, edges, w, m):
     """edges: (k, 2) int32 host array of (u, v) = v consumes u; w, m: int64 host arrays of n."""
     import numpy as np
@@ -200,6 +194,16 @@ def moc_graph_info(g):
     return dict(n=n.value, n_edges=ne.value, C=C.value, wide=bool(wide.value))
 
 
+def _check_outputs(lens, outs):
+    """The C ABI cannot see device buffer sizes: a short output would be overrun by the kernel."""
+    B = lens.numel()
+    for name, t in outs:
+        if t.numel() < B:
+            raise ValueError(f"{name} has {t.numel()} entries, the batch has {B} sequences")
+        if t.device != lens.device:
+            raise ValueError(f"{name} is on {t.device}, lens on {lens.device}")
+
+
 def moc_eval_batch(g, seqs, lens, M, out_peak=None, out_dur=None, out_feasible=None):
     """Device tensors in, device tensors out (allocated with torch if not given). Asynchronous."""
     import torch
@@ -210,6 +214,7 @@ def moc_eval_batch(g, seqs, lens, M, out_peak=None, out_dur=None, out_feasible=N
         out_dur = torch.empty(B, dtype=torch.int64, device=lens.device)
     if out_feasible is None:
         out_feasible = torch.empty(B, dtype=torch.int32, device=lens.device)
+    _check_outputs(lens, (("out_peak", out_peak), ("out_dur", out_dur), ("out_feasible", out_feasible)))
     rc = lib.moc_eval_batch(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"), B, int(M),
                             _dev(out_peak, torch.int64, "out_peak"), _dev(out_dur, torch.int64, "out_dur"),
                             _dev(out_feasible, torch.int32, "out_feasible"), _stream())
@@ -225,6 +230,7 @@ def moc_eval_batch_noalloc(g, seqs, lens, M, out_peak, out_dur, out_feasible):
     in, and the library keeps its packing offsets in a fixed array of its own device image (at most
     MOC_NOALLOC_MAX_B sequences per call; calls on one device must not overlap on the GPU)."""
     import torch
+    _check_outputs(lens, (("out_peak", out_peak), ("out_dur", out_dur), ("out_feasible", out_feasible)))
     rc = lib.moc_eval_batch_noalloc(g, _dev(seqs, torch.int32, "seqs"), _dev(lens, torch.int32, "lens"),
                                     lens.numel(), int(M), _dev(out_peak, torch.int64, "out_peak"),
                                     _dev(out_dur, torch.int64, "out_dur"),
@@ -377,6 +383,10 @@ class Graph:
 
     def info(self):
         return moc_graph_info(self.h)
+
+    def set_max_copies(self, C):
+        moc_graph_set_max_copies(self.h, C)
+        self.C = int(C)
 
     def set_caps(self, caps):
         if caps is not None and len(caps) != self.n:

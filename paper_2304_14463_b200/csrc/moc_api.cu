@@ -809,6 +809,7 @@ int moc_graph_set_max_copies(moc_graph* g, int32_t C) {
         if (rc != MOC_OK) return rc;
     }
     g->C = C;
+    ++g->generation;
     g->plan_eval.valid = false;
     g->plan_profile.valid = false;
     return MOC_OK;
@@ -851,6 +852,7 @@ int moc_graph_set_node_caps(moc_graph* g, const int32_t* caps) {
     } catch (const std::bad_alloc&) {
         return fail(MOC_ERR_NOMEM, "host allocation failed");
     }
+    ++g->generation;
     if (caps) {
         if (!g->d_cap) MOC_CUDA(cudaMalloc((void**)&g->d_cap, std::max<size_t>((size_t)g->n * 4, 16)));
         MOC_CUDA(cudaMemcpy(g->d_cap, caps, (size_t)g->n * 4, cudaMemcpyHostToDevice));

@@ -8,6 +8,7 @@ struct moc_cache {
     int device = 0;
     int32_t max_parents = 0;
     bool wide = false;
+    uint64_t graph_generation = 0;   // moc_graph::generation at the last full build
     char* d_block = nullptr;
     int64_t* d_offs = nullptr;     // max_parents + 1
     moc::EditCacheDev c{};

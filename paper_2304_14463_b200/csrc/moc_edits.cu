@@ -15,6 +15,10 @@ namespace moc_host {
 int cache_prepare(moc_cache* h, const int32_t* seqs, const int32_t* lens, const int64_t* offs, int32_t P,
                   const int32_t* todo, const int32_t* todo_count, int64_t M, int64_t* out_peak, int64_t* out_dur,
                   int32_t* out_status, cudaStream_t st) {
+    if (todo && h->graph_generation != h->g->generation)
+        return fail(MOC_ERR_ARG, "the graph's C or node caps changed after the cache was built: rebuild the cache");
+    if (h->g->C != h->c.C) return fail(MOC_ERR_ARG, "the graph's C changed after the cache was created: create a new cache");
+    if (!todo) h->graph_generation = h->g->generation;
     h->c.P = P;
     h->c.cap = h->g->d_cap;
     moc::PrepParams p{};
@@ -139,6 +143,9 @@ int moc_eval_edits(const moc_cache* h, const int32_t* parent, const int32_t* op,
     if (B == 0) return MOC_OK;
     if (!parent || !op || !q || !j || !out_peak || !out_dur || !out_status) return fail(MOC_ERR_ARG, "moc_eval_edits: null array");
     if (h->c.P < 1) return fail(MOC_ERR_ARG, "moc_eval_edits: the cache holds no parents (call moc_cache_build first)");
+    if (h->graph_generation != h->g->generation)
+        return fail(MOC_ERR_ARG, "moc_eval_edits: the graph's C or node caps changed after the cache was built "
+                    "(its copy of the caps is stale): rebuild the cache with moc_cache_build");
     DeviceGuard dg(h->device);
     if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", h->device);
     moc::EditParams p{};

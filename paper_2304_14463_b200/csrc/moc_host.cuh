@@ -87,6 +87,7 @@ struct moc_graph {
     int32_t n = 0;
     int64_t n_edges = 0;  // distinct
     int32_t C = 2;
+    uint64_t generation = 0;  // bumped whenever C or the per-node caps change: caches built before are stale
     int device = 0;
     int sm_count = 0;
     size_t smem_optin = 0;

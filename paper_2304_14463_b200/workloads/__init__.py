@@ -200,6 +200,12 @@ _SPECS = [
 N_CONFIGS = len(_SPECS)
 
 
+def budget_from_peak(peak: int, pct: int) -> int:
+    """M = floor(peak * pct / 100): a budget given as a percentage of a no-rematerialization peak
+    (Section 4.3; the budgets printed there equal this rounding of a common integer peak)."""
+    return int(peak) * int(pct) // 100
+
+
 def spec(idx):
     return dict(_SPECS[idx])
 

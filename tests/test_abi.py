@@ -7,6 +7,8 @@ import re
 import numpy as np
 import pytest
 
+from paper_2304_14463_b200 import workloads
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -93,7 +95,7 @@ def test_no_device_is_an_error_not_a_fallback(binding):
     assert rc in (-5, -6) and not h.value           # MOC_ERR_CUDA: no CPU path behind the ABI
 
 
-def test_budget_rounding_matches_printed_budgets(binding):
+def test_budget_rounding_matches_printed_budgets():
     """M = floor(P0*pct/100) reproduces the budgets printed under the plots of Section 4.3."""
     path = os.path.join(ROOT, "tests", "golden", "budget_rounding.txt")
     rows = [l for l in open(path) if l.strip() and not l.startswith("#")]
@@ -101,4 +103,4 @@ def test_budget_rounding_matches_printed_budgets(binding):
     for line in rows:
         p0 = int(line.split(":")[1].split("|")[0])
         budgets = [int(x) for x in line.split("|")[1].split()]
-        assert [binding.budget_from_peak(p0, pct) for pct in (90, 85, 80, 75)] == budgets
+        assert [workloads.budget_from_peak(p0, pct) for pct in (90, 85, 80, 75)] == budgets

@@ -149,3 +149,37 @@ def test_edits_node_caps_and_wide(B):
     # 64-bit sums
     wl.m = wl.m * (1 << 33)
     run_case(B, wl, seqs, lens, M * (1 << 33), *random_edits(rng, lens, 4000), what="wide")
+
+
+def test_stale_cache_is_refused(B):
+    """Caps or C changed after the build: the cache's copy is stale, edits are refused until a rebuild,
+    and after the rebuild they follow the new caps."""
+    wl = W.make(1, seed=4, B=32)
+    rng = np.random.default_rng(8)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    rows = [list(range(wl.n)) for _ in range(32)]
+    seqs = np.array([x for r in rows for x in r], np.int32)
+    lens = np.array([len(r) for r in rows], np.int32)
+    parent, op, q, j = random_edits(rng, lens, 3000)
+    cache = B.EditCache(G, len(lens))
+    cache.build(dev(seqs), dev(lens), M)
+    cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    caps = np.where(rng.random(wl.n) < 0.5, 1, 2).astype(np.int32)
+    for change in (lambda: G.set_caps(caps), lambda: G.set_caps(None), lambda: G.set_max_copies(2)):
+        change()
+        with pytest.raises(B.MocError, match="rebuild"):
+            cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+        cache.build(dev(seqs), dev(lens), M)
+        cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    # with the caps in force after a rebuild the results are the oracle's for those caps
+    G.set_caps(caps)
+    O.set_caps(caps)
+    cache.build(dev(seqs), dev(lens), M)
+    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    torch.cuda.synchronize()
+    got = np.stack([got[0].cpu().numpy(), got[1].cpu().numpy(), got[2].cpu().numpy().astype(np.int64)], 1)
+    want = reference(O, seqs, lens, parent, op, q, j, M, O.eval_batch(seqs, lens, M)[2])
+    assert (got == want).all()
+    torch.cuda.synchronize()

@@ -78,7 +78,7 @@ def test_config_parity_mutated(B, idx, seed):
     peaks = O.eval_batch(seqs, lens, BIG)[0]
     median = int(np.median(peaks[peaks >= 0]))
     seen = set()
-    for M in [B.budget_from_peak(P0, p) for p in wl.budget_pcts] + [P0, median]:
+    for M in [W.budget_from_peak(P0, p) for p in wl.budget_pcts] + [P0, median]:
         _, _, st = assert_batch_equal(G, O, seqs, lens, M, f"{wl.name} seed {seed} M {M}")
         seen |= set(np.unique(st).tolist())
     assert {-2, 0, 1} <= seen and (idx == 4 or -1 in seen)
@@ -92,7 +92,7 @@ def test_config_parity_full_size(B, idx):
     G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
     P0 = G.no_remat_peak()
     for pct in wl.budget_pcts:
-        assert_batch_equal(G, O, wl.seqs, wl.lens, B.budget_from_peak(P0, pct), f"{wl.name} {pct}%")
+        assert_batch_equal(G, O, wl.seqs, wl.lens, W.budget_from_peak(P0, pct), f"{wl.name} {pct}%")
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
@@ -152,7 +152,7 @@ def test_kernel_families_agree_with_oracle(B, idx, kind):
     O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
     G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
     G.set_kernel({"group": B.MOC_KERNEL_GROUP, "warp": B.MOC_KERNEL_WARP, "lane": B.MOC_KERNEL_LANE}[kind])
-    assert_batch_equal(G, O, wl.seqs, wl.lens, B.budget_from_peak(G.no_remat_peak(), 80), f"{kind} {wl.name}")
+    assert_batch_equal(G, O, wl.seqs, wl.lens, W.budget_from_peak(G.no_remat_peak(), 80), f"{kind} {wl.name}")
     assert B.moc_last_launch_count() >= 1
 
 
