@@ -33,12 +33,34 @@ METRIC = "schedule_steps_per_s_n442_B16384"
 UNIT = "steps/s"
 PCT = 80
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the evaluation kernel, from
-# one ncu capture with flushed caches (None when the kernel changed after the capture)
-NCU_TRAFFIC_BYTES = 34867200
-# executed warp instructions of the same launch (smsp__inst_executed.sum of that capture)
-NCU_WARP_INSTRUCTIONS = 34807562
-NCU_TRAFFIC_SOURCE = "ncu --set full, one launch: dram read 34.87 MB, write 0 (the 0.33 MB of results were still in L2)"
+# One ncu capture of a full-size launch of the evaluation kernel (flushed caches): DRAM traffic
+# (dram__bytes_read.sum + dram__bytes_write.sum) and executed warp instructions (smsp__inst_executed.sum),
+# valid for the kernel source whose hash is recorded with them; printed as null once the source differs.
+NCU_CAPTURE = {
+    "traffic_bytes": 34883584,
+    "warp_instructions": 29312076,
+    "source": "ncu --set full, one launch of eval_pair_kernel<int, 5>: dram read 34.88 MB, write 0 "
+              "(the 0.33 MB of results were still in L2)",
+    "kernel_sha256": "",
+}
+KERNEL_SOURCES = ["paper_2304_14463_b200/csrc/moc_pair_kernel.cuh"]
+
+
+def kernel_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def workload_config(base, M, ring_len, ring_bytes):
+    """The `config` object of the JSON line; both arms print exactly this for the same workload."""
+    return {"workload": f"{base.name}: n={base.n} m={len(base.edges)} B={base.B} C={base.C} "
+                        f"M={PCT}% of no-remat peak ({M})",
+            "sum_T_per_step": int(base.total_steps), "per_gpu_batch": int(base.B),
+            "cold_l2": f"ring of {ring_len} distinct batches, {ring_bytes / 1e6:.0f} MB of inputs > {L2_BYTES / 1e6:.0f} MB L2"}
 
 
 def load_peaks():
@@ -117,34 +139,37 @@ def make_ring(workloads, n_batches, rank, idx=WORKLOAD_IDX):
 
 
 def run_reference(args):
-    """The CPU oracle, as it stands, on the host cores: a bounded sample of the same workload."""
+    """The CPU oracle, as it stands, on the host cores: a bounded sample of the same workload (the same
+    ring of batches as the GPU arm; every step evaluates one whole batch)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2304_14463_b200 import workloads
     from oracle import OracleGraph
-    base = workloads.make(WORKLOAD_IDX, seed=1)
+    base, ring = make_ring(workloads, args.ring, 0, args.workload)
+    ring_bytes = sum(4 * int(l.sum()) + 4 * len(l) for _, l in ring)
     O = OracleGraph(base.n, base.edges, base.w, base.m, base.C)
     cores = len(os.sched_getaffinity(0))
     P0 = O.eval(np.arange(base.n), 1 << 62)["peak"]
-    M = P0 * PCT // 100
-    for _ in range(args.warmup):
-        O.eval_batch(base.seqs, base.lens, M, n_threads=cores)
+    M = workloads.budget_from_peak(P0, PCT)
+    for i in range(args.warmup):
+        O.eval_batch(ring[i % len(ring)][0], ring[i % len(ring)][1], M, n_threads=cores)
     t0 = time.perf_counter()
-    used = cores
-    for _ in range(args.steps):
-        _, _, _, used = O.eval_batch(base.seqs, base.lens, M, n_threads=cores)
+    used, steps = cores, 0
+    for i in range(args.steps):
+        seqs, lens = ring[i % len(ring)]
+        _, _, _, used = O.eval_batch(seqs, lens, M, n_threads=cores)
+        steps += int(lens.sum())
     dt = time.perf_counter() - t0
-    steps = base.total_steps * args.steps
     value = steps / dt
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+    line = {"impl": "reference", "metric": METRIC if args.workload == WORKLOAD_IDX else f"schedule_steps_per_s_{base.name}",
+            "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
             "data": "synthetic",
-            "config": {"workload": f"{base.name}: n={base.n} m={len(base.edges)} B={base.B} C={base.C} "
-                                   f"M={PCT}% of no-remat peak", "sum_T": base.total_steps},
+            "config": workload_config(base, M, len(ring), ring_bytes),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle",
-                             "sample": f"the full batch ({base.B} sequences, {base.total_steps} steps) per step, "
+                             "sample": f"one whole batch ({base.B} sequences, about {base.total_steps} steps) per step, "
                                        f"{args.steps} steps"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -527,19 +552,33 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident throughput: K steps back to back on one stream
+    # ---- device-resident throughput: K steps back to back on one stream.  A short region (the
+    # driver's --steps 20 is about a millisecond) is repeated and the median region reported, so
+    # that one slow launch does not decide the figure and the clock sampler sees the GPU under load.
     for i in range(args.warmup):
         step(i)
     launches_per_step = binding.moc_last_launch_count()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(min(args.steps, 20)):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    est_ms = e0.elapsed_time(e1) / min(args.steps, 20) * args.steps
+    repeats = 1 if est_ms >= 100.0 else int(min(200, max(25, 100.0 / max(est_ms, 1e-3))))
+    barrier()
+    region_ms = []
     with ClockSampler(local_rank) as clocks:
-        e0.record(stream)
-        for i in range(args.steps):
-            step(i)
-        e1.record(stream)
-        barrier()
-    ms = e0.elapsed_time(e1)
+        for r in range(repeats):
+            e0.record(stream)
+            for i in range(args.steps):
+                step(r * args.steps + i)
+            e1.record(stream)
+            barrier()
+            region_ms.append(e0.elapsed_time(e1))
+    ms = float(np.median(region_ms))
+    # every region runs the same number of steps over the ring; count the steps of the median-length one
     steps_done = sum(ring[i % len(ring)]["steps"] for i in range(args.steps))
 
     # ---- the same region again with the library's measurement hook: an event pair around every
@@ -585,6 +624,17 @@ def main():
                        dur=torch.empty(B, dtype=torch.int64).pin_memory(),
                        st=torch.empty(B, dtype=torch.int32).pin_memory(), steps=int(lens.sum()), B=B))
     n_e2e = max(3, min(args.steps, 64))
+    # pinned host -> device bandwidth of this machine for the same bytes: what the end-to-end figures are bound by
+    d_tmp = torch.empty_like(hr[0]["seqs"], device="cuda")
+    for _ in range(3):
+        d_tmp.copy_(hr[0]["seqs"], non_blocking=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(10):
+        d_tmp.copy_(hr[0]["seqs"], non_blocking=True)
+    torch.cuda.synchronize()
+    link_gbs = 10 * hr[0]["seqs"].numel() * 4 / (time.perf_counter() - t0) / 1e9
+    del d_tmp
     for i in range(3):
         r = hr[i % len(hr)]
         G.eval_batch_host(r["seqs"], r["lens"], M, r["peak"], r["dur"], r["st"])
@@ -629,6 +679,8 @@ def main():
         r0 = ring[0]
         alg_bytes = 4 * r0["steps"] + 4 * r0["B"] + 20 * r0["B"]
         kernel_ms = float(np.mean(kern_ms))
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        capture_ok = args.workload == WORKLOAD_IDX and NCU_CAPTURE["kernel_sha256"] == kernel_sha256()
         if launches_per_step == 1:
             # one kernel per step: the timed region itself (K back-to-back launches between two CUDA
             # events) is the cleaner per-launch figure; the per-launch event pairs add record overhead
@@ -639,40 +691,39 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64" if info["wide"] else "int32", "data": "synthetic",
-            "config": {"workload": f"{base.name}: n={base.n} m={len(base.edges)} B={base.B} C={base.C} "
-                                   f"M={PCT}% of no-remat peak ({M})",
-                       "sum_T_per_step": r0["steps"], "cold_l2": f"ring of {len(ring)} distinct batches, "
-                       f"{ring_bytes / 1e6:.0f} MB of inputs > {L2_BYTES / 1e6:.0f} MB L2",
-                       "per_gpu_batch": base.B},
+            "config": workload_config(base, M, len(ring), ring_bytes),
+            "timed_regions": repeats, "region_ms_median_min_max": [ms, float(np.min(region_ms)), float(np.max(region_ms))],
             "gpu_launches": launches_per_step * args.steps,
             "e2e": {"value": e2e_steps / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": 4 * hr[0]["steps"] + 4 * hr[0]["B"], "d2h_bytes_per_step": 20 * hr[0]["B"],
-                    "steps": n_e2e, "api": "moc_eval_batch_host (pinned host buffers)"},
+                    "steps": n_e2e, "api": "moc_eval_batch_host (pinned host buffers)", "link_gbs": link_gbs,
+                    "link_frac": (4 * hr[0]["steps"] + 4 * hr[0]["B"]) / (e2e_s / n_e2e) / 1e9 / link_gbs},
             "e2e_u16": None if e2e16_s is None else {
                 "value": e2e16_steps / e2e16_s, "unit": UNIT, "h2d_bytes_per_step": 2 * hr[0]["steps"] + 4 * hr[0]["B"],
                 "d2h_bytes_per_step": 20 * hr[0]["B"], "steps": n_e2e,
-                "api": "moc_eval_batch_host16 (node ids as uint16 in pinned host buffers)"},
+                "api": "moc_eval_batch_host16 (node ids as uint16 in pinned host buffers)", "link_gbs": link_gbs,
+                "link_frac": (2 * hr[0]["steps"] + 4 * hr[0]["B"]) / (e2e16_s / n_e2e) / 1e9 / link_gbs},
             "roofline": {"bound": "hbm", "achieved": alg_bytes / (kernel_ms * 1e-3) / 1e9, "peak": peak_gbs,
                          "unit": "GB/s", "frac": alg_bytes / (kernel_ms * 1e-3) / 1e9 / peak_gbs,
                          "peak_kind": f"of {peak_kind}",
-                         "traffic": NCU_TRAFFIC_BYTES if args.workload == WORKLOAD_IDX else None,
-                         "traffic_source": NCU_TRAFFIC_SOURCE if args.workload == WORKLOAD_IDX else None,
+                         "traffic": NCU_CAPTURE["traffic_bytes"] if capture_ok else None,
+                         "traffic_source": NCU_CAPTURE["source"] if capture_ok else
+                                           "no capture of this kernel source and workload (the recorded one is stale)",
                          "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": kernel_ms,
                          "kernel": "evaluation kernel (CUDA events around each launch, mean of %d)" % n_k,
                          "between_kernels_ms": float(np.mean(gap_ms)),
                          "graph_replay_ms_per_step": graph_ms,
-                         "note": "the kernel is bound by shared-memory wavefronts and instruction issue, "
-                                 "not by HBM (ncu: issue slots 71 %, ALU pipe 57 %, shared-memory data pipe 67 %, DRAM 9 % busy)"},
+                         "note": "the kernel is bound on chip (shared-memory data pipe, instruction issue), not by HBM: see profiles/"},
             "clocks": clocks.summary(),
         }
-        if args.workload == WORKLOAD_IDX:
-            # Second view of the same launch: the limit ncu shows is instruction issue and the integer /
-            # shared-memory pipes.  Issue peak = SMs x 4 schedulers x 1 warp instruction per clock.
+        if capture_ok:
+            # Second view of the same launch: the limits ncu shows are instruction issue and the shared-memory
+            # pipe.  Issue peak = SMs x 4 schedulers x 1 warp instruction per clock.
             sm_mhz = line["clocks"]["sm_mhz"] or 1965.0
-            issue_peak = 148 * 4 * sm_mhz * 1e6
-            line["issue_roofline"] = {"bound": "alu", "achieved": NCU_WARP_INSTRUCTIONS / (kernel_ms * 1e-3) / 1e9,
+            issue_peak = sm_count * 4 * sm_mhz * 1e6
+            line["issue_roofline"] = {"bound": "alu", "achieved": NCU_CAPTURE["warp_instructions"] / (kernel_ms * 1e-3) / 1e9,
                                       "peak": issue_peak / 1e9, "unit": "G warp instructions/s",
-                                      "frac": NCU_WARP_INSTRUCTIONS / (kernel_ms * 1e-3) / issue_peak,
+                                      "frac": NCU_CAPTURE["warp_instructions"] / (kernel_ms * 1e-3) / issue_peak,
                                       "note": "executed (not algorithmic) instructions of one launch from the ncu capture; "
                                               "context for the HBM fraction above, not a replacement"}
         if not args.no_cpu_baseline:

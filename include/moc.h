@@ -123,7 +123,10 @@ int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens,
  * Same evaluation with every array in HOST memory (pinned memory makes the copies asynchronous
  * with respect to the host, pageable memory works too): copies seqs (n_steps ints, which must be
  * at least sum(max(lens[b],0))) and lens to device staging owned by the handle, evaluates, copies
- * the three outputs back and synchronises `stream` before returning.
+ * the three outputs back and synchronises `stream` before returning.  Large batches travel in up
+ * to eight chunks of whole sequences: a copy stream owned by the handle brings one chunk while
+ * `stream` evaluates the one before, and the results return in a single copy through a pinned
+ * block of the handle.  One call at a time per handle.
  */
 int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps,
                         const int32_t* lens, int32_t B, int64_t M, int64_t* out_peak,
@@ -401,7 +404,8 @@ int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t seq
 
 /*
  * Which evaluation kernel moc_eval_batch uses, and in what shape.  The library has three families
- * for the operation of Section 2 (Eqs. 1-8); all give the same results, and MOC_KERNEL_AUTO (the
+ * for the operation of Section 2 (Eqs. 1-8) -- four with the packed variant for up to four copies --;
+ * all give the same results, and MOC_KERNEL_AUTO (the
  * default) picks the fastest one that can serve the graph.  The call exists so that tests can
  * compare every family with the oracle and so that launch shapes can be measured.
  *   MOC_KERNEL_AUTO   a = b = 0.
@@ -411,6 +415,9 @@ int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t seq
  *   MOC_KERNEL_LANE   one sequence per lane: a block keeps a group of a sequences (0, 8, 16, 32)
  *                     on chip and its b warps (0, 8, 16, 24 or 32; a multiple of a) share the work on them;
  *                     C <= 2 and a graph whose state for a group fits in shared memory.
+ *   MOC_KERNEL_BLOCK  one block of a threads (0, or a multiple of 32 in 64..1024) per sequence with
+ *                     the copies of a node packed into one 64-bit word, b = 0; C <= 4 and sequences
+ *                     of at most 32766 steps whose state fits in shared memory.
  * MOC_ERR_ARG for an unknown kind or shape; a kind that cannot serve the graph with its current C
  * is reported by the next moc_eval_batch (MOC_ERR_ARG), which evaluates nothing.
  */
@@ -418,6 +425,7 @@ int moc_graph_set_launch(moc_graph* g, int32_t threads_per_sequence, int32_t seq
 #define MOC_KERNEL_GROUP 1
 #define MOC_KERNEL_WARP 2
 #define MOC_KERNEL_LANE 3
+#define MOC_KERNEL_BLOCK 4
 int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b);
 
 /*

@@ -164,7 +164,7 @@ def moc_graph_set_launch(g, threads_per_sequence=0, sequences_per_block=0):
            "moc_graph_set_launch")
 
 
-MOC_KERNEL_AUTO, MOC_KERNEL_GROUP, MOC_KERNEL_WARP, MOC_KERNEL_LANE = 0, 1, 2, 3
+MOC_KERNEL_AUTO, MOC_KERNEL_GROUP, MOC_KERNEL_WARP, MOC_KERNEL_LANE, MOC_KERNEL_BLOCK = 0, 1, 2, 3, 4
 
 
 def moc_graph_set_kernel(g, kind=MOC_KERNEL_AUTO, a=0, b=0):

@@ -97,6 +97,11 @@ LaneFn lane_fn_lg(int lg, int kp) {
 }
 LaneFn lane_fn(bool wide, int lg, int kp) { return wide ? lane_fn_lg<int64_t>(lg, kp) : lane_fn_lg<int32_t>(lg, kp); }
 
+QuadFn quad_fn(bool wide, int C) {
+    if (C <= 3) return wide ? (QuadFn)moc::eval_quad_kernel<int64_t, 3> : (QuadFn)moc::eval_quad_kernel<int32_t, 3>;
+    return wide ? (QuadFn)moc::eval_quad_kernel<int64_t, 4> : (QuadFn)moc::eval_quad_kernel<int32_t, 4>;
+}
+
 // Raises a kernel's dynamic shared-memory limit to all the device offers beside its static part.
 cudaError_t raise_smem_limit(const void* fn, size_t smem_optin) {
     cudaFuncAttributes a{};
@@ -167,6 +172,37 @@ const char* plan_lane(const moc_graph* g, size_t smem_cap, Plan* out) {
     return "the state of a group of sequences exceeds shared memory in the requested shape, n >= 4096, or a degree above 255";
 }
 
+// Plan of the block-per-sequence path with packed words (C <= 4).  Returns nullptr on success.
+const char* plan_quad(const moc_graph* g, size_t smem_cap, Plan* out) {
+    Plan pl = *out;
+    const int64_t n = g->n, C = g->C, t_max = C * n;
+    if (C > 4) return "C > 4";
+    if (!g->d_order) return "n above 32000 or a degree above 65535";
+    if (t_max > 32766) return "sequences of more than 32766 steps";
+    const size_t msz = pl.wide ? 8 : 4;
+    const size_t word_b = align16(8 * (size_t)(n + 2)), cnt_b = align16(2 * (size_t)(n + 2)), delta_b = align16(msz * (size_t)(t_max + 4));
+    const size_t sm = word_b + cnt_b + delta_b;
+    if (sm > smem_cap) return "the state of a sequence exceeds shared memory";
+    QuadFn fn = quad_fn(pl.wide, (int)C);
+    if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); return "cudaFuncSetAttribute failed"; }
+    // threads: about one per four nodes, a power of two in [128, 1024]; or as requested
+    int thr = g->want_kind == MOC_KERNEL_BLOCK && g->want_a ? g->want_a : std::min(1024, std::max(128, pow2_ceil((int)(n / 4))));
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, thr, sm) != cudaSuccess || nb < 1) { cudaGetLastError(); return "kernel does not fit on an SM"; }
+    pl.quad = true;
+    pl.quad_fn = fn;
+    pl.G = thr;
+    pl.gpc = 1;
+    pl.block = thr;
+    pl.smem = sm;
+    pl.grid = g->sm_count * nb;
+    pl.quad_word_b = (uint32_t)word_b;
+    pl.quad_cnt_b = (uint32_t)cnt_b;
+    pl.valid = true;
+    *out = pl;
+    return nullptr;
+}
+
 // Chooses kernel variant, group size and grid for the handle's current n and C.  The dynamic
 // shared-memory limit of a kernel is a property of the kernel, not of the handle: it is always
 // raised to the device maximum, so that handles with different needs can share one kernel.
@@ -194,6 +230,14 @@ int make_plan(const moc_graph* g, bool profile, Plan* out) {
             return MOC_OK;
         }
         if (kind == MOC_KERNEL_LANE) return fail(MOC_ERR_ARG, "the sequence-per-lane kernel cannot serve this graph: %s", why);
+    }
+    if (kind == MOC_KERNEL_BLOCK || (kind == MOC_KERNEL_AUTO && !shape_given && !profile && C >= 3)) {
+        const char* why = plan_quad(g, smem_cap, &pl);
+        if (!why) {
+            *out = pl;
+            return MOC_OK;
+        }
+        if (kind == MOC_KERNEL_BLOCK) return fail(MOC_ERR_ARG, "the block-per-sequence kernel cannot serve this graph: %s", why);
     }
     if (kind == MOC_KERNEL_WARP && !warp_ok)
         return fail(MOC_ERR_ARG, "the warp-per-sequence kernel cannot serve this graph (C > 2, degrees too uneven or C * sum(w) >= 2^48)");
@@ -402,6 +446,31 @@ int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, con
     return upload_lane_rec(g);
 }
 
+// Layout for the block-per-sequence kernel: the nodes in order of falling out-degree (a sink counts one:
+// its made-up successor n + 1) with the place of their successor lists, and the lists as 16-bit ids.
+int build_quad_layout(moc_graph* g, const std::vector<int32_t>& succ_start, const std::vector<int32_t>& succ) {
+    const int32_t n = g->n;
+    if (n > 32000) return MOC_OK;
+    auto deg = [&](int32_t v) { return std::max(1, succ_start[v + 1] - succ_start[v]); };
+    std::vector<int32_t> order((size_t)n);
+    for (int32_t v = 0; v < n; ++v) order[v] = v;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
+    if (deg(order[0]) > 65535) return MOC_OK;
+    std::vector<uint2> rec((size_t)n);
+    std::vector<uint16_t> ids;
+    for (int32_t i = 0; i < n; ++i) {
+        const int32_t v = order[i];
+        rec[i] = make_uint2((uint32_t)v | ((uint32_t)deg(v) << 16), (uint32_t)ids.size());
+        if (succ_start[v + 1] == succ_start[v]) ids.push_back((uint16_t)(n + 1));
+        for (int32_t e = succ_start[v]; e < succ_start[v + 1]; ++e) ids.push_back((uint16_t)succ[e]);
+    }
+    MOC_CUDA(cudaMalloc((void**)&g->d_order, rec.size() * sizeof(uint2)));
+    MOC_CUDA(cudaMalloc((void**)&g->d_succ16, std::max<size_t>(ids.size() * 2, 16)));
+    MOC_CUDA(cudaMemcpy(g->d_order, rec.data(), rec.size() * sizeof(uint2), cudaMemcpyHostToDevice));
+    MOC_CUDA(cudaMemcpy(g->d_succ16, ids.data(), ids.size() * 2, cudaMemcpyHostToDevice));
+    return MOC_OK;
+}
+
 moc::EvalParams base_params(const moc_graph* g, const Plan& pl) {
     moc::EvalParams p{};
     p.g.n = g->n;
@@ -463,7 +532,28 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    if (pl.lane) {
+    if (pl.quad) {
+        moc::QuadParams q{};
+        q.n = g->n;
+        q.C = g->C;
+        q.max_T = g->C * g->n;
+        q.B = B;
+        q.M = M;
+        q.order = g->d_order;
+        q.succ = g->d_succ16;
+        q.m = pl.wide ? (const void*)g->d_m64 : (const void*)g->d_m32;
+        q.w = g->d_w;
+        q.cap = g->d_cap;
+        q.seqs = seqs;
+        q.lens = lens;
+        q.offs = offs;
+        q.out_peak = out_peak;
+        q.out_dur = out_dur;
+        q.out_status = out_feasible;
+        q.word_bytes = pl.quad_word_b;
+        q.cnt_bytes = pl.quad_cnt_b;
+        MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.quad_fn, q));
+    } else if (pl.lane) {
         const LaneLayout& L = g->lane[5 - pl.lane_lg];
         moc::LaneParams q{};
         q.n = g->n;
@@ -789,6 +879,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     try {
         rc = build_lane_layouts(g, succ_start, succ, m, m32);
         if (rc == MOC_OK) rc = upload_wslot(g);
+        if (rc == MOC_OK) rc = build_quad_layout(g, succ_start, succ);
     } catch (const std::bad_alloc&) {
         rc = fail(MOC_ERR_NOMEM, "host allocation failed");
     }
@@ -876,6 +967,7 @@ int moc_graph_set_kernel(moc_graph* g, int32_t kind, int32_t a, int32_t b) {
                  !(a && b && a * b > 1024);
             break;
         case MOC_KERNEL_WARP: ok = a == 0 && (b == 0 || (b >= 4 && b <= 16)); break;
+        case MOC_KERNEL_BLOCK: ok = (a == 0 || (a >= 64 && a <= 1024 && a % 32 == 0)) && b == 0; break;
         case MOC_KERNEL_LANE: ok = (a == 0 || a == 8 || a == 16 || a == 32) && (b == 0 || (b >= 8 && b <= 32 && b % 8 == 0)); break;
         default: break;
     }
@@ -931,6 +1023,13 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_stage_seqs);
     cudaFree(g->d_stage_u16);
     cudaFree(g->d_stage_io);
+    cudaFree(g->d_order);
+    cudaFree(g->d_succ16);
+    if (g->h_stage) cudaFreeHost(g->h_stage);
+    if (g->copy_stream) {
+        cudaStreamDestroy(g->copy_stream);
+        for (cudaEvent_t ev : g->chunk_ev) cudaEventDestroy(ev);
+    }
     for (int li = 0; li < 3; ++li) {
         cudaFree(g->lane[li].d_rec32);
         cudaFree(g->lane[li].d_rec64);
@@ -963,6 +1062,109 @@ int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens,
     return launch_eval(g, seqs, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream);
 }
 
+// Host entry points.  The batch is cut into chunks of whole sequences; a copy stream owned by the
+// handle brings chunk k + 1 to the device while the caller's stream evaluates chunk k (one
+// cudaMemcpyAsync per chunk and an event between the two streams), and the three result arrays come
+// back with one copy into a pinned staging block, from which they are handed to the caller's arrays.
+namespace {
+constexpr int kHostChunks = 8;
+
+int host_streams(const moc_graph* g) {
+    if (g->copy_stream) return MOC_OK;
+    MOC_CUDA(cudaStreamCreateWithFlags(&g->copy_stream, cudaStreamNonBlocking));
+    for (int k = 0; k < kHostChunks + 1; ++k) MOC_CUDA(cudaEventCreateWithFlags(&g->chunk_ev[k], cudaEventDisableTiming));
+    return MOC_OK;
+}
+
+// ids: host array of `need` node ids, 4 bytes each (wide_ids) or 2 bytes each.
+int eval_host(const moc_graph* g, const void* ids, bool wide_ids, int64_t n_steps, const int32_t* lens, int32_t B,
+              int64_t M, int64_t* out_peak, int64_t* out_dur, int32_t* out_feasible, cudaStream_t st, const char* who) {
+    // chunk boundaries: about equal numbers of steps, whole sequences
+    int64_t need = 0;
+    for (int32_t b = 0; b < B; ++b) need += lens[b] > 0 ? lens[b] : 0;
+    if (need > n_steps) return fail(MOC_ERR_ARG, "%s: lens sum to %lld > n_steps %lld", who, (long long)need, (long long)n_steps);
+    int32_t cb[kHostChunks + 1];
+    int64_t co[kHostChunks + 1];
+    int n_chunks = 0;
+    {
+        const int want = (int)std::max<int64_t>(1, std::min<int64_t>(kHostChunks, need / (1 << 18)));   // at least a MB of ids per chunk
+        int64_t run = 0;
+        cb[0] = 0;
+        co[0] = 0;
+        for (int32_t b = 0; b < B; ++b) {
+            run += lens[b] > 0 ? lens[b] : 0;
+            if (n_chunks + 1 < want && run >= need * (n_chunks + 1) / want) {
+                ++n_chunks;
+                cb[n_chunks] = b + 1;
+                co[n_chunks] = run;
+            }
+        }
+        ++n_chunks;
+        cb[n_chunks] = B;
+        co[n_chunks] = need;
+    }
+    DeviceGuard dg(g->device);
+    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
+    int rc = host_streams(g);
+    if (rc != MOC_OK) return rc;
+    rc = ensure((void**)&g->d_stage_seqs, &g->stage_seqs_cap, std::max<size_t>((size_t)need * 4 + 16, 16));
+    if (rc != MOC_OK) return rc;
+    if (!wide_ids) {
+        rc = ensure((void**)&g->d_stage_u16, &g->stage_u16_cap, std::max<size_t>((size_t)need * 2 + 16, 16));
+        if (rc != MOC_OK) return rc;
+    }
+    const size_t bB = (size_t)B, o_peak = 0, o_dur = bB * 8, o_st = 2 * bB * 8, o_lens = align16(o_st + bB * 4),
+                 res_bytes = o_st + bB * 4, io_bytes = o_lens + bB * 4;
+    rc = ensure((void**)&g->d_stage_io, &g->stage_io_cap, io_bytes);
+    if (rc != MOC_OK) return rc;
+    if (res_bytes > g->h_stage_cap) {
+        if (g->h_stage) MOC_CUDA(cudaFreeHost(g->h_stage));
+        g->h_stage = nullptr;
+        g->h_stage_cap = 0;
+        MOC_CUDA(cudaMallocHost((void**)&g->h_stage, res_bytes * 2));
+        g->h_stage_cap = res_bytes * 2;
+    }
+    int64_t* d_peak = (int64_t*)(g->d_stage_io + o_peak);
+    int64_t* d_dur = (int64_t*)(g->d_stage_io + o_dur);
+    int32_t* d_st = (int32_t*)(g->d_stage_io + o_st);
+    int32_t* d_lens = (int32_t*)(g->d_stage_io + o_lens);
+    cudaStream_t cs = g->copy_stream;
+    // the copy stream starts once the caller's stream has reached this call
+    MOC_CUDA(cudaEventRecord(g->chunk_ev[kHostChunks], st));
+    MOC_CUDA(cudaStreamWaitEvent(cs, g->chunk_ev[kHostChunks], 0));
+    MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, cs));
+    int launches = 0;
+    for (int k = 0; k < n_chunks; ++k) {
+        const int64_t s0 = co[k], cnt = co[k + 1] - co[k];
+        if (cnt) {
+            if (wide_ids)
+                MOC_CUDA(cudaMemcpyAsync(g->d_stage_seqs + s0, (const int32_t*)ids + s0, (size_t)cnt * 4, cudaMemcpyHostToDevice, cs));
+            else
+                MOC_CUDA(cudaMemcpyAsync(g->d_stage_u16 + s0, (const uint16_t*)ids + s0, (size_t)cnt * 2, cudaMemcpyHostToDevice, cs));
+        }
+        MOC_CUDA(cudaEventRecord(g->chunk_ev[k], cs));
+        MOC_CUDA(cudaStreamWaitEvent(st, g->chunk_ev[k], 0));
+        if (cnt && !wide_ids) {
+            const int blocks = (int)std::min<int64_t>((cnt / 8 + 255) / 256 + 1, (int64_t)g->sm_count * 8);
+            moc::widen_ids_kernel<<<blocks, 256, 0, st>>>(g->d_stage_u16 + s0, g->d_stage_seqs + s0, cnt);
+            ++launches;
+        }
+        const int32_t b0 = cb[k], nb = cb[k + 1] - cb[k];
+        if (nb > 0) {
+            rc = launch_eval(g, g->d_stage_seqs + s0, d_lens + b0, nb, M, d_peak + b0, d_dur + b0, d_st + b0, st);
+            if (rc != MOC_OK) return rc;
+        }
+    }
+    g_launches += launches;      // the evaluation launches were counted as they were enqueued
+    MOC_CUDA(cudaMemcpyAsync(g->h_stage, g->d_stage_io, res_bytes, cudaMemcpyDeviceToHost, st));
+    MOC_CUDA(cudaStreamSynchronize(st));
+    memcpy(out_peak, g->h_stage + o_peak, bB * 8);
+    memcpy(out_dur, g->h_stage + o_dur, bB * 8);
+    memcpy(out_feasible, g->h_stage + o_st, bB * 4);
+    return MOC_OK;
+}
+}  // namespace
+
 int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps, const int32_t* lens,
                         int32_t B, int64_t M, int64_t* out_peak, int64_t* out_dur,
                         int32_t* out_feasible, void* stream) {
@@ -972,31 +1174,7 @@ int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps
     if (B == 0) return MOC_OK;
     if (!lens || !out_peak || !out_dur || !out_feasible || (n_steps > 0 && !seqs))
         return fail(MOC_ERR_ARG, "moc_eval_batch_host: null array");
-    int64_t need = 0;
-    for (int32_t b = 0; b < B; ++b) need += lens[b] > 0 ? lens[b] : 0;
-    if (need > n_steps) return fail(MOC_ERR_ARG, "moc_eval_batch_host: lens sum to %lld > n_steps %lld", (long long)need, (long long)n_steps);
-    DeviceGuard dg(g->device);
-    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
-    cudaStream_t st = (cudaStream_t)stream;
-    int rc = ensure((void**)&g->d_stage_seqs, &g->stage_seqs_cap, std::max<size_t>((size_t)need * 4, 16));
-    if (rc != MOC_OK) return rc;
-    const size_t bB = (size_t)B, o_lens = 0, o_peak = align16(bB * 4), o_dur = o_peak + bB * 8,
-                 o_st = o_dur + bB * 8, io_bytes = o_st + bB * 4;
-    rc = ensure((void**)&g->d_stage_io, &g->stage_io_cap, io_bytes);
-    if (rc != MOC_OK) return rc;
-    int32_t* d_lens = (int32_t*)(g->d_stage_io + o_lens);
-    int64_t* d_peak = (int64_t*)(g->d_stage_io + o_peak);
-    int64_t* d_dur = (int64_t*)(g->d_stage_io + o_dur);
-    int32_t* d_st = (int32_t*)(g->d_stage_io + o_st);
-    if (need) MOC_CUDA(cudaMemcpyAsync(g->d_stage_seqs, seqs, (size_t)need * 4, cudaMemcpyHostToDevice, st));
-    MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, st));
-    rc = launch_eval(g, g->d_stage_seqs, d_lens, B, M, d_peak, d_dur, d_st, st);
-    if (rc != MOC_OK) return rc;
-    MOC_CUDA(cudaMemcpyAsync(out_peak, d_peak, bB * 8, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaMemcpyAsync(out_dur, d_dur, bB * 8, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaMemcpyAsync(out_feasible, d_st, bB * 4, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaStreamSynchronize(st));
-    return MOC_OK;
+    return eval_host(g, seqs, true, n_steps, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream, "moc_eval_batch_host");
 }
 
 int moc_eval_batch_host16(const moc_graph* g, const uint16_t* seqs, int64_t n_steps, const int32_t* lens,
@@ -1009,38 +1187,7 @@ int moc_eval_batch_host16(const moc_graph* g, const uint16_t* seqs, int64_t n_st
     if (B == 0) return MOC_OK;
     if (!lens || !out_peak || !out_dur || !out_feasible || (n_steps > 0 && !seqs))
         return fail(MOC_ERR_ARG, "moc_eval_batch_host16: null array");
-    int64_t need = 0;
-    for (int32_t b = 0; b < B; ++b) need += lens[b] > 0 ? lens[b] : 0;
-    if (need > n_steps) return fail(MOC_ERR_ARG, "moc_eval_batch_host16: lens sum to %lld > n_steps %lld", (long long)need, (long long)n_steps);
-    DeviceGuard dg(g->device);
-    if (!dg.ok) return fail(MOC_ERR_CUDA, "cannot select device %d", g->device);
-    cudaStream_t st = (cudaStream_t)stream;
-    int rc = ensure((void**)&g->d_stage_seqs, &g->stage_seqs_cap, std::max<size_t>((size_t)need * 4, 16));
-    if (rc != MOC_OK) return rc;
-    rc = ensure((void**)&g->d_stage_u16, &g->stage_u16_cap, std::max<size_t>((size_t)need * 2, 16));
-    if (rc != MOC_OK) return rc;
-    const size_t bB = (size_t)B, o_lens = 0, o_peak = align16(bB * 4), o_dur = o_peak + bB * 8,
-                 o_st = o_dur + bB * 8, io_bytes = o_st + bB * 4;
-    rc = ensure((void**)&g->d_stage_io, &g->stage_io_cap, io_bytes);
-    if (rc != MOC_OK) return rc;
-    int32_t* d_lens = (int32_t*)(g->d_stage_io + o_lens);
-    int64_t* d_peak = (int64_t*)(g->d_stage_io + o_peak);
-    int64_t* d_dur = (int64_t*)(g->d_stage_io + o_dur);
-    int32_t* d_st = (int32_t*)(g->d_stage_io + o_st);
-    if (need) {
-        MOC_CUDA(cudaMemcpyAsync(g->d_stage_u16, seqs, (size_t)need * 2, cudaMemcpyHostToDevice, st));
-        const int blocks = (int)std::min<int64_t>((need / 8 + 255) / 256 + 1, (int64_t)g->sm_count * 8);
-        moc::widen_ids_kernel<<<blocks, 256, 0, st>>>(g->d_stage_u16, g->d_stage_seqs, need);
-    }
-    MOC_CUDA(cudaMemcpyAsync(d_lens, lens, bB * 4, cudaMemcpyHostToDevice, st));
-    rc = launch_eval(g, g->d_stage_seqs, d_lens, B, M, d_peak, d_dur, d_st, st);
-    if (rc != MOC_OK) return rc;
-    if (need) ++g_launches;
-    MOC_CUDA(cudaMemcpyAsync(out_peak, d_peak, bB * 8, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaMemcpyAsync(out_dur, d_dur, bB * 8, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaMemcpyAsync(out_feasible, d_st, bB * 4, cudaMemcpyDeviceToHost, st));
-    MOC_CUDA(cudaStreamSynchronize(st));
-    return MOC_OK;
+    return eval_host(g, seqs, false, n_steps, lens, B, M, out_peak, out_dur, out_feasible, (cudaStream_t)stream, "moc_eval_batch_host16");
 }
 
 // ---- evaluation without any allocation -----------------------------------------------------------

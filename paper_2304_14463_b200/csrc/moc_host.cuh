@@ -11,12 +11,14 @@
 #include "moc_kernels.cuh"
 #include "moc_pair_kernel.cuh"
 #include "moc_lane_kernel.cuh"
+#include "moc_quad_kernel.cuh"
 
 namespace moc_host {
 
 using KernelFn = void (*)(const moc::EvalParams);
 using PairFn = void (*)(const moc::PairParams);
 using LaneFn = void (*)(const moc::LaneParams);
+using QuadFn = void (*)(const moc::QuadParams);
 
 struct Plan {
     bool valid = false;
@@ -33,6 +35,10 @@ struct Plan {
     int pair_nb[17] = {0};
     size_t pair_graph_b = 0, pair_warp_b = 0;
     int sm_count = 0;
+    // block-per-sequence path with packed words for C <= 4
+    bool quad = false;
+    QuadFn quad_fn = nullptr;
+    uint32_t quad_word_b = 0, quad_cnt_b = 0;
     // sequence-per-lane path for C <= 2: a block keeps a group of 8, 16 or 32 sequences on chip
     bool lane = false;
     LaneFn lane_fn = nullptr;
@@ -104,6 +110,8 @@ struct moc_graph {
     int32_t want_G = 0, want_gpc = 0;
     int32_t want_kind = 0, want_a = 0, want_b = 0;   // moc_graph_set_kernel
     moc_host::LaneLayout lane[3];         // groups of 32, 16, 8 sequences
+    uint2* d_order = nullptr;             // block-per-sequence kernel: nodes by falling out-degree {node | degree << 16, first entry}
+    uint16_t* d_succ16 = nullptr;         // ... and their successor ids (a sink: n + 1)
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
     // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
     int32_t sell_len = 0, n_tiles = 0;
@@ -125,8 +133,12 @@ struct moc_graph {
     mutable size_t stage_seqs_cap = 0;
     mutable uint16_t* d_stage_u16 = nullptr;   // 16-bit node ids as they arrive from the host
     mutable size_t stage_u16_cap = 0;
-    mutable char* d_stage_io = nullptr;  // lens | peak | dur | status
+    mutable char* d_stage_io = nullptr;  // peak | dur | status | lens
     mutable size_t stage_io_cap = 0;
+    mutable char* h_stage = nullptr;     // pinned: peak | dur | status as they come back in one copy
+    mutable size_t h_stage_cap = 0;
+    mutable cudaStream_t copy_stream = nullptr;   // host entry points: brings the next chunk while one is evaluated
+    mutable cudaEvent_t chunk_ev[9] = {};
 };
 
 

@@ -144,16 +144,59 @@ def test_lane_kernel_shapes(B, idx, a, b):
     assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), f"lane {a}x{b} {wl.name}")
 
 
-@pytest.mark.parametrize("kind", ["group", "warp", "lane"])
+@pytest.mark.parametrize("kind", ["group", "warp", "lane", "block"])
 @pytest.mark.parametrize("idx", [0, 1, 2])
 def test_kernel_families_agree_with_oracle(B, idx, kind):
-    """Each family forced in turn on the full batch of the configurations all three can serve."""
+    """Each family forced in turn on the full batch of the configurations all of them can serve."""
     wl = W.make(idx, seed=2)
     O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
     G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
-    G.set_kernel({"group": B.MOC_KERNEL_GROUP, "warp": B.MOC_KERNEL_WARP, "lane": B.MOC_KERNEL_LANE}[kind])
+    G.set_kernel({"group": B.MOC_KERNEL_GROUP, "warp": B.MOC_KERNEL_WARP, "lane": B.MOC_KERNEL_LANE,
+                  "block": B.MOC_KERNEL_BLOCK}[kind])
     assert_batch_equal(G, O, wl.seqs, wl.lens, W.budget_from_peak(G.no_remat_peak(), 80), f"{kind} {wl.name}")
     assert B.moc_last_launch_count() >= 1
+
+
+@pytest.mark.parametrize("idx", range(W.N_CONFIGS))
+@pytest.mark.parametrize("threads", [0, 64, 160, 1024])
+def test_block_kernel_shapes(B, idx, threads):
+    """The block-per-sequence kernel with packed words on damaged batches of every configuration (C = 2 and 3),
+    with few and many threads per sequence."""
+    wl = W.make(idx, seed=8, B=[300, 400, 200, 96, 24][idx])
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G.set_kernel(B.MOC_KERNEL_BLOCK, threads, 0)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=6, frac=1 / 8)
+    peaks = O.eval_batch(seqs, lens, BIG)[0]
+    _, _, st = assert_batch_equal(G, O, seqs, lens, int(np.median(peaks[peaks >= 0])), f"block {threads} {wl.name}")
+    assert {0, 1} <= set(st.tolist()) and (idx == 4 or -2 in st)
+
+
+@pytest.mark.parametrize("C", [1, 2, 3, 4])
+def test_block_kernel_every_cap_and_wide(B, C):
+    """Caps 1..4, per-node caps, and sums that need 64 bits, on sequences with up to four copies per node."""
+    wl = W.make(1, seed=3, B=64)
+    rng = np.random.default_rng(C)
+    rows = []
+    for _ in range(200):
+        r = list(rng.permutation(wl.n)) if rng.random() < 0.1 else list(range(wl.n))
+        for v in range(wl.n):
+            for _ in range(int(rng.integers(0, 5)) if rng.random() < 0.15 else 0):
+                r.insert(int(rng.integers(r.index(v) + 1, len(r) + 1)), v)
+        rows.append(r)
+    seqs, lens = W.pack(rows)
+    for scale, caps in ((1, None), (1 << 26, None), (1, np.asarray(rng.integers(1, C + 1, wl.n), np.int32))):
+        m = wl.m * scale
+        O = OracleGraph(wl.n, wl.edges, wl.w, m, C)
+        G = B.Graph(wl.n, wl.edges, wl.w, m, C)
+        if caps is not None:
+            O.set_caps(caps)
+            G.set_caps(caps)
+        G.set_kernel(B.MOC_KERNEL_BLOCK)
+        peaks = O.eval_batch(seqs, lens, BIG)[0]
+        M = int(np.median(peaks[peaks >= 0])) if (peaks >= 0).any() else 1
+        _, _, st = assert_batch_equal(G, O, seqs, lens, M, f"block C={C} scale={scale} caps={caps is not None}")
+    assert G.info()["wide"] is False or scale > 1
 
 
 def test_lane_kernel_refuses_what_it_cannot_serve(B):
@@ -365,6 +408,32 @@ def test_host_entry_point_u16(B):
     p2, d2, s2 = np.empty(len(lens), np.int64), np.empty(len(lens), np.int64), np.empty(len(lens), np.int32)
     G.eval_batch_host16(buf[1:], lens, M, p2, d2, s2)
     assert (p2 == op).all() and (d2 == od).all() and (s2 == os_).all()
+
+
+def test_host_entry_points_in_chunks(B):
+    """A batch large enough to travel in several chunks (copy of one chunk under the evaluation of the
+    one before), cut at sequence boundaries that do not divide the batch evenly; damaged sequences and
+    a zero-length one sit at chunk edges like anywhere else."""
+    wl = W.make(2, seed=11, B=5003)
+    O = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    G = B.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    seqs, lens = W.mutate(wl.seqs, wl.lens, wl.n, wl.C, seed=3, frac=1 / 8)
+    seqs = np.where(seqs < 0, 65535, seqs).astype(np.int32)
+    M = O.eval(np.arange(wl.n), BIG)["peak"] * 80 // 100
+    op, od, os_, _ = O.eval_batch(seqs, lens, M)
+    l = torch.from_numpy(lens).pin_memory()
+    outs = [torch.empty(len(lens), dtype=dt).pin_memory() for dt in (torch.int64, torch.int64, torch.int32)]
+    for rep in range(2):
+        G.eval_batch_host(torch.from_numpy(seqs).pin_memory(), l, M, *outs)
+        assert B.moc_last_launch_count() >= 4
+        assert (outs[0].numpy() == op).all() and (outs[1].numpy() == od).all() and (outs[2].numpy() == os_).all()
+        for o in outs:
+            o.zero_()
+        G.eval_batch_host16(torch.from_numpy(seqs.astype(np.uint16)).pin_memory(), l, M, *outs)
+        assert B.moc_last_launch_count() >= 8
+        assert (outs[0].numpy() == op).all() and (outs[1].numpy() == od).all() and (outs[2].numpy() == os_).all()
+    # the device entry point on the same handle in between is not disturbed
+    assert_batch_equal(G, O, seqs[:int(np.clip(lens[:100], 0, None).sum())], lens[:100], M, "after host calls")
 
 
 def test_state_in_global_memory(B):
