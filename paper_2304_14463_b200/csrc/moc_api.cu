@@ -177,16 +177,18 @@ const char* plan_quad(const moc_graph* g, size_t smem_cap, Plan* out) {
     Plan pl = *out;
     const int64_t n = g->n, C = g->C, t_max = C * n;
     if (C > 4) return "C > 4";
-    if (!g->d_order) return "n above 32000 or a degree above 65535";
+    if (!g->d_order32) return "n above 32000 or a degree above 65535";
     if (t_max > 32766) return "sequences of more than 32766 steps";
     const size_t msz = pl.wide ? 8 : 4;
     const size_t word_b = align16(8 * (size_t)(n + 2)), cnt_b = align16(2 * (size_t)(n + 2)), delta_b = align16(msz * (size_t)(t_max + 4));
-    const size_t sm = word_b + cnt_b + delta_b;
+    // a copy of m per block where it costs little next to the state
+    const size_t m_b = 4 * (word_b + cnt_b + delta_b + msz * (size_t)n) <= smem_cap ? align16(msz * (size_t)n) : 0;
+    const size_t sm = word_b + cnt_b + m_b + delta_b;
     if (sm > smem_cap) return "the state of a sequence exceeds shared memory";
     QuadFn fn = quad_fn(pl.wide, (int)C);
     if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); return "cudaFuncSetAttribute failed"; }
-    // threads: about one per four nodes, a power of two in [128, 1024]; or as requested
-    int thr = g->want_kind == MOC_KERNEL_BLOCK && g->want_a ? g->want_a : std::min(1024, std::max(128, pow2_ceil((int)(n / 4))));
+    // threads: a warp per 280 nodes or so (measured: 4 warps at n = 1000, 18 at n = 5000), or as requested
+    int thr = g->want_kind == MOC_KERNEL_BLOCK && g->want_a ? g->want_a : 32 * (int)std::min<int64_t>(32, std::max<int64_t>(2, (n + 140) / 280));
     int nb = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, thr, sm) != cudaSuccess || nb < 1) { cudaGetLastError(); return "kernel does not fit on an SM"; }
     pl.quad = true;
@@ -198,6 +200,7 @@ const char* plan_quad(const moc_graph* g, size_t smem_cap, Plan* out) {
     pl.grid = g->sm_count * nb;
     pl.quad_word_b = (uint32_t)word_b;
     pl.quad_cnt_b = (uint32_t)cnt_b;
+    pl.quad_m_b = (uint32_t)m_b;
     pl.valid = true;
     *out = pl;
     return nullptr;
@@ -448,7 +451,8 @@ int build_lane_layouts(moc_graph* g, const std::vector<int32_t>& succ_start, con
 
 // Layout for the block-per-sequence kernel: the nodes in order of falling out-degree (a sink counts one:
 // its made-up successor n + 1) with the place of their successor lists, and the lists as 16-bit ids.
-int build_quad_layout(moc_graph* g, const std::vector<int32_t>& succ_start, const std::vector<int32_t>& succ) {
+int build_quad_layout(moc_graph* g, const std::vector<int32_t>& succ_start, const std::vector<int32_t>& succ,
+                      const int64_t* m, const std::vector<int32_t>& m32) {
     const int32_t n = g->n;
     if (n > 32000) return MOC_OK;
     auto deg = [&](int32_t v) { return std::max(1, succ_start[v + 1] - succ_start[v]); };
@@ -456,18 +460,36 @@ int build_quad_layout(moc_graph* g, const std::vector<int32_t>& succ_start, cons
     for (int32_t v = 0; v < n; ++v) order[v] = v;
     std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return deg(x) > deg(y); });
     if (deg(order[0]) > 65535) return MOC_OK;
-    std::vector<uint2> rec((size_t)n);
-    std::vector<uint16_t> ids;
-    for (int32_t i = 0; i < n; ++i) {
-        const int32_t v = order[i];
-        rec[i] = make_uint2((uint32_t)v | ((uint32_t)deg(v) << 16), (uint32_t)ids.size());
-        if (succ_start[v + 1] == succ_start[v]) ids.push_back((uint16_t)(n + 1));
-        for (int32_t e = succ_start[v]; e < succ_start[v + 1]; ++e) ids.push_back((uint16_t)succ[e]);
+    for (int wide = 0; wide < 2; ++wide) {
+        std::vector<uint32_t> rec((size_t)n * 8, 0u);
+        std::vector<uint16_t> rest;
+        for (int32_t i = 0; i < n; ++i) {
+            const int32_t v = order[i];
+            std::vector<uint16_t> ids;
+            if (succ_start[v + 1] == succ_start[v]) ids.push_back((uint16_t)(n + 1));
+            for (int32_t e = succ_start[v]; e < succ_start[v + 1]; ++e) ids.push_back((uint16_t)succ[e]);
+            uint32_t* r = &rec[(size_t)i * 8];
+            r[0] = (uint32_t)v | ((uint32_t)ids.size() << 16);
+            r[1] = (uint32_t)rest.size();
+            if (wide) {
+                r[2] = (uint32_t)((uint64_t)m[v] & 0xFFFFFFFFu);
+                r[3] = (uint32_t)((uint64_t)m[v] >> 32);
+            } else {
+                r[2] = (uint32_t)m32[v];
+            }
+            for (size_t k = 0; k < ids.size(); ++k) {
+                if (k < 8) r[4 + k / 2] |= (uint32_t)ids[k] << (16 * (k & 1));
+                else rest.push_back(ids[k]);
+            }
+        }
+        uint4** dst = wide ? &g->d_order64 : &g->d_order32;
+        MOC_CUDA(cudaMalloc((void**)dst, rec.size() * 4));
+        MOC_CUDA(cudaMemcpy(*dst, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice));
+        if (!wide) {
+            MOC_CUDA(cudaMalloc((void**)&g->d_succ16, std::max<size_t>(rest.size() * 2, 16)));
+            if (!rest.empty()) MOC_CUDA(cudaMemcpy(g->d_succ16, rest.data(), rest.size() * 2, cudaMemcpyHostToDevice));
+        }
     }
-    MOC_CUDA(cudaMalloc((void**)&g->d_order, rec.size() * sizeof(uint2)));
-    MOC_CUDA(cudaMalloc((void**)&g->d_succ16, std::max<size_t>(ids.size() * 2, 16)));
-    MOC_CUDA(cudaMemcpy(g->d_order, rec.data(), rec.size() * sizeof(uint2), cudaMemcpyHostToDevice));
-    MOC_CUDA(cudaMemcpy(g->d_succ16, ids.data(), ids.size() * 2, cudaMemcpyHostToDevice));
     return MOC_OK;
 }
 
@@ -539,7 +561,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.max_T = g->C * g->n;
         q.B = B;
         q.M = M;
-        q.order = g->d_order;
+        q.order = pl.wide ? g->d_order64 : g->d_order32;
         q.succ = g->d_succ16;
         q.m = pl.wide ? (const void*)g->d_m64 : (const void*)g->d_m32;
         q.w = g->d_w;
@@ -552,6 +574,7 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.out_status = out_feasible;
         q.word_bytes = pl.quad_word_b;
         q.cnt_bytes = pl.quad_cnt_b;
+        q.m_bytes = pl.quad_m_b;
         MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.quad_fn, q));
     } else if (pl.lane) {
         const LaneLayout& L = g->lane[5 - pl.lane_lg];
@@ -879,7 +902,7 @@ int moc_graph_create(int32_t n, int64_t n_edges, const int32_t* edges, const int
     try {
         rc = build_lane_layouts(g, succ_start, succ, m, m32);
         if (rc == MOC_OK) rc = upload_wslot(g);
-        if (rc == MOC_OK) rc = build_quad_layout(g, succ_start, succ);
+        if (rc == MOC_OK) rc = build_quad_layout(g, succ_start, succ, m, m32);
     } catch (const std::bad_alloc&) {
         rc = fail(MOC_ERR_NOMEM, "host allocation failed");
     }
@@ -1023,7 +1046,8 @@ void moc_graph_destroy(moc_graph* g) {
     cudaFree(g->d_stage_seqs);
     cudaFree(g->d_stage_u16);
     cudaFree(g->d_stage_io);
-    cudaFree(g->d_order);
+    cudaFree(g->d_order32);
+    cudaFree(g->d_order64);
     cudaFree(g->d_succ16);
     if (g->h_stage) cudaFreeHost(g->h_stage);
     if (g->copy_stream) {

@@ -38,7 +38,7 @@ struct Plan {
     // block-per-sequence path with packed words for C <= 4
     bool quad = false;
     QuadFn quad_fn = nullptr;
-    uint32_t quad_word_b = 0, quad_cnt_b = 0;
+    uint32_t quad_word_b = 0, quad_cnt_b = 0, quad_m_b = 0;
     // sequence-per-lane path for C <= 2: a block keeps a group of 8, 16 or 32 sequences on chip
     bool lane = false;
     LaneFn lane_fn = nullptr;
@@ -110,8 +110,9 @@ struct moc_graph {
     int32_t want_G = 0, want_gpc = 0;
     int32_t want_kind = 0, want_a = 0, want_b = 0;   // moc_graph_set_kernel
     moc_host::LaneLayout lane[3];         // groups of 32, 16, 8 sequences
-    uint2* d_order = nullptr;             // block-per-sequence kernel: nodes by falling out-degree {node | degree << 16, first entry}
-    uint16_t* d_succ16 = nullptr;         // ... and their successor ids (a sink: n + 1)
+    uint4* d_order32 = nullptr;           // block-per-sequence kernel: 32-byte node records by falling out-degree (32- / 64-bit m)
+    uint4* d_order64 = nullptr;
+    uint16_t* d_succ16 = nullptr;         // ... and the successors beyond a node's eighth
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // measurement hook around the evaluation kernel
     // sliced-ELL successor lists in out-degree order (null when the fast path cannot serve the graph)
     int32_t sell_len = 0, n_tiles = 0;

@@ -45,8 +45,8 @@ struct QuadParams {
     int32_t max_T;             // C * n
     int32_t B;
     int64_t M;
-    const uint2* order;        // n records in order of falling out-degree: {node | out-degree << 16 (a sink: 1), first successor entry}
-    const uint16_t* succ;      // successor node ids grouped by producer (a sink: the id n + 1)
+    const uint4* order;        // n records of 32 bytes in order of falling out-degree (below)
+    const uint16_t* succ;      // the successors beyond the eighth of the nodes that have more
     const void* m;             // n output sizes, int32 or int64
     const int64_t* w;          // n durations
     const int32_t* cap;        // n per-node caps, or nullptr
@@ -58,7 +58,12 @@ struct QuadParams {
     int32_t* out_status;
     uint32_t word_bytes;       // 8 (n + 2), rounded to 16
     uint32_t cnt_bytes;        // 2 (n + 2), rounded to 16
+    uint32_t m_bytes;          // sizeof(sum) * n rounded to 16 when the block keeps a copy of m in shared memory, else 0
 };
+
+// Node record: word 0 = node | out-degree << 16 (a sink: 1, its successor the id n + 1), word 1 = index
+// of its ninth successor in `succ`, words 2-3 = m (int32: word 2), words 4-7 = its first eight successor
+// ids, 16 bits each.
 
 __device__ __forceinline__ void sts_u64(uint32_t addr, uint64_t v) {
     asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
@@ -94,11 +99,17 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
     int n = p.n;
     MOC_KEEP(n);
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
-    uint32_t wa = sbase, ca = sbase + p.word_bytes, da = ca + p.cnt_bytes;   // words | counters | delta[0..]
+    uint32_t wa = sbase, ca = sbase + p.word_bytes, ma = ca + p.cnt_bytes, da = ma + p.m_bytes;   // words | counters | m | delta[0..]
     MOC_KEEP(wa);
     MOC_KEEP(ca);
+    MOC_KEEP(ma);
     MOC_KEEP(da);
     const MemT* gm = reinterpret_cast<const MemT*>(p.m);
+    const bool m_on_chip = p.m_bytes != 0;
+    if (m_on_chip) {
+        for (int i = tid; i < n; i += nthr) sts_mem(ma + ((uint32_t)i << kShift), __ldg(gm + i));
+        __syncthreads();
+    }
 
     for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
         const int64_t off = __ldg(p.offs + b);
@@ -119,18 +130,27 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
             uint32_t flags = 0;    // bit 0: malformed, bit 1: precedence violated
             {
                 const int32_t* row = p.seqs + off;
-                for (int t = tid; t < T; t += nthr) {
-                    const uint32_t id = (uint32_t)__ldg(row + t);
+                auto put = [&](uint32_t id, int t) {
                     if (id < (uint32_t)n) {
                         const uint32_t sh = (id & 1u) << 4;
                         const uint32_t k = (atom_add_shared_u32(ca + ((id >> 1) << 2), 1u << sh) >> sh) & 0xFFFFu;
                         if (k < 4) sts_u16(wa + (id << 3) + (k << 1), (uint32_t)t + 1u);
-                        sts_mem(da + ((uint32_t)t << kShift), __ldg(gm + id));
+                        sts_mem(da + ((uint32_t)t << kShift), m_on_chip ? lds_mem(ma + (id << kShift), MemT()) : __ldg(gm + id));
                     } else {
                         flags = 1;
                         sts_mem(da + ((uint32_t)t << kShift), MemT(0));
                     }
+                };
+                int t = tid;
+                for (; t + 3 * nthr < T; t += 4 * nthr) {      // four loads in flight per thread
+                    const uint32_t i0 = (uint32_t)__ldg(row + t), i1 = (uint32_t)__ldg(row + t + nthr),
+                                   i2 = (uint32_t)__ldg(row + t + 2 * nthr), i3 = (uint32_t)__ldg(row + t + 3 * nthr);
+                    put(i0, t);
+                    put(i1, t + nthr);
+                    put(i2, t + 2 * nthr);
+                    put(i3, t + 3 * nthr);
                 }
+                for (; t < T; t += nthr) put((uint32_t)__ldg(row + t), t);
                 if (tid == 0) sts_u64(wa + ((uint32_t)(n + 1) << 3), (uint64_t)(uint32_t)T * 0x0001000100010001ull);
             }
             __syncthreads();
@@ -165,12 +185,17 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
                 uint32_t depw = 0;
                 const int n_round = (n + 31) & ~31;
                 for (int i = tid; i < n_round; i += nthr) {
-                    uint32_t node = 0, deg = 0, e0 = 0;
+                    uint32_t node = 0, deg = 0, e8 = 0;
+                    uint4 inl = make_uint4(0, 0, 0, 0);
+                    MemT neg_m = 0;
                     if (i < n) {
-                        const uint2 r = __ldg(p.order + i);
+                        const uint4 r = __ldg(p.order + 2 * i);
+                        inl = __ldg(p.order + 2 * i + 1);
                         node = r.x & 0xFFFFu;
                         deg = r.x >> 16;
-                        e0 = r.y;
+                        e8 = r.y;
+                        if constexpr (sizeof(MemT) == 4) neg_m = -(MemT)r.z;
+                        else neg_m = -(MemT)((uint64_t)r.z | ((uint64_t)r.w << 32));
                     }
                     const int rounds = __reduce_max_sync(0xFFFFFFFFu, (int)deg);
                     const uint2 own = lds_v2(wa + (node << 3));
@@ -186,19 +211,24 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
                     G[0] = (last - base[0]) * 0x10001u;                                          // the last copy ends at itself at least
 #pragma unroll
                     for (int j = 1; j < kAcc; ++j) G[j] = ((base[j - 1] - base[j]) & 0xFFFFu) * 0x10001u;   // copy j ends at itself at least
-                    for (int k = 0; k < rounds; ++k) {
-                        if ((uint32_t)k < deg) {
-                            const uint32_t s = (uint32_t)__ldg(p.succ + e0 + k);
-                            const uint2 r = lds_v2(wa + (s << 3));
+                    auto visit = [&](uint32_t sid) {
+                        const uint2 r = lds_v2(wa + (sid << 3));
 #pragma unroll
-                            for (int j = 0; j < kAcc; ++j) {
-                                G[j] = __viaddmax_u16x2(r.x, na[j], G[j]);
-                                G[j] = __viaddmax_u16x2(r.y, na[j], G[j]);
-                            }
+                        for (int j = 0; j < kAcc; ++j) {
+                            G[j] = __viaddmax_u16x2(r.x, na[j], G[j]);
+                            G[j] = __viaddmax_u16x2(r.y, na[j], G[j]);
+                        }
+                    };
+                    const uint32_t in8[4] = {inl.x, inl.y, inl.z, inl.w};
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (k < rounds) {
+                            if ((uint32_t)k < deg) visit((k & 1) ? in8[k >> 1] >> 16 : in8[k >> 1] & 0xFFFFu);
                         }
                     }
+                    for (int k = 8; k < rounds; ++k)
+                        if ((uint32_t)k < deg) visit((uint32_t)__ldg(p.succ + e8 + (k - 8)));
                     if (i < n) {
-                        const MemT neg_m = -__ldg(gm + node);
                         const uint32_t g0 = max_halves(G[0]);
                         depw |= g0;                                           // bit 15: a successor copy before a_1
                         red_add_shared(da + (((base[0] + g0) & 0xFFFFu) << kShift), neg_m);

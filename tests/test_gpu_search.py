@@ -1,5 +1,7 @@
 """Parity of the search entry points (through the C ABI) with the search oracle: after any number of
 generations every chain's sequence, length, evaluation and acceptance count are identical."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -217,3 +219,64 @@ def test_search_incremental_errors(B):
     S3 = B.Search(G3, dev(wl3.seqs), dev(wl3.lens), 1 << 60, 1)
     with pytest.raises(B.MocError):
         S3.set_samples(2, incremental=True)
+
+
+# ------------------------------------------------------------------ a population split over two ranks
+def _rank_worker(rank, world, port, q):
+    import os
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2304_14463_b200 import binding, sharding, workloads
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    torch.cuda.set_device(0)                        # both ranks share the one GPU; nothing waits on a peer's kernel
+    wl = workloads.make(1, seed=6, B=192, n_threads=1)
+    G = binding.Graph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = workloads.budget_from_peak(G.no_remat_peak(), 85)
+    my_seqs, my_lens = sharding.shard_batch(wl.seqs, wl.lens, rank, world)
+    b0, b1 = sharding.shard_range(len(wl.lens), rank, world)
+    S = binding.Search(G, torch.from_numpy(np.ascontiguousarray(my_seqs)).cuda(), torch.from_numpy(np.ascontiguousarray(my_lens)).cuda(),
+                       M, seed=11, first_chain=b0)
+    S.run(25)
+    st = S.state()
+    torch.cuda.synchronize()
+    mine = S.best()
+    got = sharding.best_over_ranks(mine, M, b0, wl.C * wl.n)
+    lens_all = [torch.zeros(len(wl.lens), dtype=torch.int64) for _ in range(world)]
+    part = torch.zeros(len(wl.lens), dtype=torch.int64)
+    part[b0:b1] = st["lens"].cpu().to(torch.int64)
+    dist.all_gather(lens_all, part)
+    if rank == 0:
+        full = binding.Search(G, torch.from_numpy(wl.seqs).cuda(), torch.from_numpy(wl.lens).cuda(), M, seed=11)
+        full.run(25)
+        fs = full.state()
+        fb = full.best()
+        torch.cuda.synchronize()
+        same_lens = bool((sum(lens_all) == fs["lens"].cpu().to(torch.int64)).all())
+        q.put((same_lens, got["index"] == fb["index"], bool((got["seq"] == fb["seq"]).all()),
+               (got["peak"], got["dur"], got["status"]) == (fb["peak"], fb["dur"], fb["status"])))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_population_split_over_two_ranks_on_the_gpu():
+    """Two processes (gloo for the host-side exchange), each driving a CUDA search handle on its half of
+    the chains with their global chain numbers: the chains evolve exactly as in the unsplit CUDA run and
+    the best chain over the ranks is the unsplit best."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 33500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    out = q.get(timeout=300)
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    assert out == (True, True, True, True)
