@@ -123,10 +123,11 @@ int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens,
  * Same evaluation with every array in HOST memory (pinned memory makes the copies asynchronous
  * with respect to the host, pageable memory works too): copies seqs (n_steps ints, which must be
  * at least sum(max(lens[b],0))) and lens to device staging owned by the handle, evaluates, copies
- * the three outputs back and synchronises `stream` before returning.  Large batches travel in up
- * to eight chunks of whole sequences: a copy stream owned by the handle brings one chunk while
- * `stream` evaluates the one before, and the results return in a single copy through a pinned
- * block of the handle.  One call at a time per handle.
+ * the three outputs back and synchronises `stream` before returning.  Large batches travel in
+ * four chunks of whole sequences (a half, a quarter and two eighths of the steps): a copy stream
+ * owned by the handle brings one chunk while `stream` evaluates the one before, so that only the
+ * evaluation of the small last chunk is not hidden, and the results return in a single copy
+ * through a pinned block of the handle.  One call at a time per handle.
  */
 int moc_eval_batch_host(const moc_graph* g, const int32_t* seqs, int64_t n_steps,
                         const int32_t* lens, int32_t B, int64_t M, int64_t* out_peak,

@@ -1091,12 +1091,12 @@ int moc_eval_batch(const moc_graph* g, const int32_t* seqs, const int32_t* lens,
 // cudaMemcpyAsync per chunk and an event between the two streams), and the three result arrays come
 // back with one copy into a pinned staging block, from which they are handed to the caller's arrays.
 namespace {
-constexpr int kHostChunks = 8;
+constexpr int kHostChunks = 4;
 
 int host_streams(const moc_graph* g) {
     if (g->copy_stream) return MOC_OK;
     MOC_CUDA(cudaStreamCreateWithFlags(&g->copy_stream, cudaStreamNonBlocking));
-    for (int k = 0; k < kHostChunks + 1; ++k) MOC_CUDA(cudaEventCreateWithFlags(&g->chunk_ev[k], cudaEventDisableTiming));
+    for (int k = 0; k < kHostChunks + 1; ++k) MOC_CUDA(cudaEventCreateWithFlags(&g->chunk_ev[k], cudaEventDisableTiming));   // chunk_ev has room for 9
     return MOC_OK;
 }
 
@@ -1111,16 +1111,19 @@ int eval_host(const moc_graph* g, const void* ids, bool wide_ids, int64_t n_step
     int64_t co[kHostChunks + 1];
     int n_chunks = 0;
     {
-        const int want = (int)std::max<int64_t>(1, std::min<int64_t>(kHostChunks, need / (1 << 18)));   // at least a MB of ids per chunk
-        int64_t run = 0;
+        // Chunks of 1/2, 1/4, 1/8, 1/8 of the steps (whole sequences): the evaluation of all but the last
+        // chunk hides behind the copy of the next, and the last one is small.  Short batches go in one piece.
+        const int want = need >= (int64_t(1) << 21) ? kHostChunks : 1;
+        int64_t run = 0, bound = need - need / 2;
         cb[0] = 0;
         co[0] = 0;
         for (int32_t b = 0; b < B; ++b) {
             run += lens[b] > 0 ? lens[b] : 0;
-            if (n_chunks + 1 < want && run >= need * (n_chunks + 1) / want) {
+            if (n_chunks + 1 < want && run >= bound) {
                 ++n_chunks;
                 cb[n_chunks] = b + 1;
                 co[n_chunks] = run;
+                bound = run + (need - run + 1) / 2;
             }
         }
         ++n_chunks;

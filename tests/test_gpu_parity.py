@@ -425,12 +425,12 @@ def test_host_entry_points_in_chunks(B):
     outs = [torch.empty(len(lens), dtype=dt).pin_memory() for dt in (torch.int64, torch.int64, torch.int32)]
     for rep in range(2):
         G.eval_batch_host(torch.from_numpy(seqs).pin_memory(), l, M, *outs)
-        assert B.moc_last_launch_count() >= 4
+        assert B.moc_last_launch_count() >= 3
         assert (outs[0].numpy() == op).all() and (outs[1].numpy() == od).all() and (outs[2].numpy() == os_).all()
         for o in outs:
             o.zero_()
         G.eval_batch_host16(torch.from_numpy(seqs.astype(np.uint16)).pin_memory(), l, M, *outs)
-        assert B.moc_last_launch_count() >= 8
+        assert B.moc_last_launch_count() >= 6
         assert (outs[0].numpy() == op).all() and (outs[1].numpy() == od).all() and (outs[2].numpy() == os_).all()
     # the device entry point on the same handle in between is not disturbed
     assert_batch_equal(G, O, seqs[:int(np.clip(lens[:100], 0, None).sum())], lens[:100], M, "after host calls")
