@@ -489,6 +489,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", type=int, default=WORKLOAD_IDX,
                     help="index 0..4 of the configuration to time (default: the headline one)")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "group", "warp", "lane", "block"],
+                    help="evaluation kernel family to time (default: the library's own choice)")
     ap.add_argument("--mode", default="eval", choices=["eval", "search", "intervals", "edits"],
                     help="eval: the headline evaluation metric; search: generations of the search entry points; "
                          "intervals: the interval-form checker; edits: the incremental evaluation of single edits")
@@ -530,6 +532,8 @@ def main():
 
     base, ring_host = make_ring(workloads, args.ring, rank, args.workload)
     G = binding.Graph(base.n, base.edges, base.w, base.m, base.C)
+    G.set_kernel({"auto": binding.MOC_KERNEL_AUTO, "group": binding.MOC_KERNEL_GROUP, "warp": binding.MOC_KERNEL_WARP,
+                  "lane": binding.MOC_KERNEL_LANE, "block": binding.MOC_KERNEL_BLOCK}[args.kernel])
     M = workloads.budget_from_peak(G.no_remat_peak(), PCT)
     ring = []
     for seqs, lens in ring_host:
@@ -680,7 +684,7 @@ def main():
         alg_bytes = 4 * r0["steps"] + 4 * r0["B"] + 20 * r0["B"]
         kernel_ms = float(np.mean(kern_ms))
         sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
-        capture_ok = args.workload == WORKLOAD_IDX and NCU_CAPTURE["kernel_sha256"] == kernel_sha256()
+        capture_ok = args.workload == WORKLOAD_IDX and args.kernel == "auto" and NCU_CAPTURE["kernel_sha256"] == kernel_sha256()
         if launches_per_step == 1:
             # one kernel per step: the timed region itself (K back-to-back launches between two CUDA
             # events) is the cleaner per-launch figure; the per-launch event pairs add record overhead
@@ -691,7 +695,7 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64" if info["wide"] else "int32", "data": "synthetic",
-            "config": workload_config(base, M, len(ring), ring_bytes),
+            "config": workload_config(base, M, len(ring), ring_bytes), "kernel_family": args.kernel,
             "timed_regions": repeats, "region_ms_median_min_max": [ms, float(np.min(region_ms)), float(np.max(region_ms))],
             "gpu_launches": launches_per_step * args.steps,
             "e2e": {"value": e2e_steps / e2e_s, "unit": UNIT,

@@ -181,14 +181,14 @@ const char* plan_quad(const moc_graph* g, size_t smem_cap, Plan* out) {
     if (t_max > 32766) return "sequences of more than 32766 steps";
     const size_t msz = pl.wide ? 8 : 4;
     const size_t word_b = align16(8 * (size_t)(n + 2)), cnt_b = align16(2 * (size_t)(n + 2)), delta_b = align16(msz * (size_t)(t_max + 4));
-    // a copy of m per block where it costs little next to the state
-    const size_t m_b = 4 * (word_b + cnt_b + delta_b + msz * (size_t)n) <= smem_cap ? align16(msz * (size_t)n) : 0;
-    const size_t sm = word_b + cnt_b + m_b + delta_b;
+    const size_t sm = word_b + cnt_b + delta_b;
     if (sm > smem_cap) return "the state of a sequence exceeds shared memory";
     QuadFn fn = quad_fn(pl.wide, (int)C);
     if (raise_smem_limit((const void*)fn, g->smem_optin) != cudaSuccess) { cudaGetLastError(); return "cudaFuncSetAttribute failed"; }
-    // threads: a warp per 280 nodes or so (measured: 4 warps at n = 1000, 18 at n = 5000), or as requested
-    int thr = g->want_kind == MOC_KERNEL_BLOCK && g->want_a ? g->want_a : 32 * (int)std::min<int64_t>(32, std::max<int64_t>(2, (n + 140) / 280));
+    // threads per sequence, from measurements at n = 100, 1000 and 5000 (more threads lose to the block-wide
+    // barriers, fewer to the length of the per-thread loops); or as requested
+    int thr = n < 200 ? 64 : (n < 1600 ? 128 : (n < 12000 ? 512 : 1024));
+    if (g->want_kind == MOC_KERNEL_BLOCK && g->want_a) thr = g->want_a;
     int nb = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, thr, sm) != cudaSuccess || nb < 1) { cudaGetLastError(); return "kernel does not fit on an SM"; }
     pl.quad = true;
@@ -200,7 +200,6 @@ const char* plan_quad(const moc_graph* g, size_t smem_cap, Plan* out) {
     pl.grid = g->sm_count * nb;
     pl.quad_word_b = (uint32_t)word_b;
     pl.quad_cnt_b = (uint32_t)cnt_b;
-    pl.quad_m_b = (uint32_t)m_b;
     pl.valid = true;
     *out = pl;
     return nullptr;
@@ -574,7 +573,6 @@ int enqueue_eval(const moc_graph* g, const Plan& pl, int64_t* offs, bool fill_of
         q.out_status = out_feasible;
         q.word_bytes = pl.quad_word_b;
         q.cnt_bytes = pl.quad_cnt_b;
-        q.m_bytes = pl.quad_m_b;
         MOC_CUDA(cudaLaunchKernelEx(&cfg, pl.quad_fn, q));
     } else if (pl.lane) {
         const LaneLayout& L = g->lane[5 - pl.lane_lg];

@@ -38,7 +38,7 @@ struct Plan {
     // block-per-sequence path with packed words for C <= 4
     bool quad = false;
     QuadFn quad_fn = nullptr;
-    uint32_t quad_word_b = 0, quad_cnt_b = 0, quad_m_b = 0;
+    uint32_t quad_word_b = 0, quad_cnt_b = 0;
     // sequence-per-lane path for C <= 2: a block keeps a group of 8, 16 or 32 sequences on chip
     bool lane = false;
     LaneFn lane_fn = nullptr;

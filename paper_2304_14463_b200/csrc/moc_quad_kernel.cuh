@@ -11,11 +11,12 @@
 //
 // Stages for one sequence seq[0..T) (paper: Section 2, Eqs. 1-8):
 //   1a. occurrence words  step t takes the next free quarter of its node's word (a 16-bit counter per
-//                         node, two counters per 32-bit atomic) and stores t + 1 there; it also
-//                         writes delta[t] = m of its node ("+m at the copy's own step" of stage 3).
+//                         node, two counters per 32-bit atomic) and stores t + 1 there.
 //   1b. per node          count in [1, min(C, C_v)] (Eq. 7 and the cap), duration += count * w
 //                         (Eq. 1); the quarters are sorted with a five-comparator network on packed
-//                         halves (empty quarters last) and the empty ones filled with the last copy.
+//                         halves (empty quarters last) and the empty ones filled with the last copy;
+//                         delta[p - 1] = m for every copy p ("+m at the copy's own step" of stage 3:
+//                         a plain store, every step belongs to exactly one copy).
 //   2.  free steps        one thread per node u with copies a_1 <= ... <= a_4, nodes taken in order of
 //                         falling out-degree so that the lanes of a warp run about the same number of
 //                         rounds; per successor word r (both halves, two packed operations each):
@@ -58,7 +59,6 @@ struct QuadParams {
     int32_t* out_status;
     uint32_t word_bytes;       // 8 (n + 2), rounded to 16
     uint32_t cnt_bytes;        // 2 (n + 2), rounded to 16
-    uint32_t m_bytes;          // sizeof(sum) * n rounded to 16 when the block keeps a copy of m in shared memory, else 0
 };
 
 // Node record: word 0 = node | out-degree << 16 (a sink: 1, its successor the id n + 1), word 1 = index
@@ -99,17 +99,11 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
     int n = p.n;
     MOC_KEEP(n);
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
-    uint32_t wa = sbase, ca = sbase + p.word_bytes, ma = ca + p.cnt_bytes, da = ma + p.m_bytes;   // words | counters | m | delta[0..]
+    uint32_t wa = sbase, ca = sbase + p.word_bytes, da = ca + p.cnt_bytes;   // words | counters | delta[0..]
     MOC_KEEP(wa);
     MOC_KEEP(ca);
-    MOC_KEEP(ma);
     MOC_KEEP(da);
     const MemT* gm = reinterpret_cast<const MemT*>(p.m);
-    const bool m_on_chip = p.m_bytes != 0;
-    if (m_on_chip) {
-        for (int i = tid; i < n; i += nthr) sts_mem(ma + ((uint32_t)i << kShift), __ldg(gm + i));
-        __syncthreads();
-    }
 
     for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
         const int64_t off = __ldg(p.offs + b);
@@ -135,10 +129,8 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
                         const uint32_t sh = (id & 1u) << 4;
                         const uint32_t k = (atom_add_shared_u32(ca + ((id >> 1) << 2), 1u << sh) >> sh) & 0xFFFFu;
                         if (k < 4) sts_u16(wa + (id << 3) + (k << 1), (uint32_t)t + 1u);
-                        sts_mem(da + ((uint32_t)t << kShift), m_on_chip ? lds_mem(ma + (id << kShift), MemT()) : __ldg(gm + id));
                     } else {
                         flags = 1;
-                        sts_mem(da + ((uint32_t)t << kShift), MemT(0));
                     }
                 };
                 int t = tid;
@@ -171,6 +163,17 @@ __global__ void __launch_bounds__(1024) eval_quad_kernel(const QuadParams p) {
                 lo = __viaddmax_u16x2(min_u16x2(lo, cap_key), 0x00010001u, 0u);        // back to positions, empties = last copy
                 hi = __viaddmax_u16x2(min_u16x2(hi, cap_key), 0x00010001u, 0u);
                 sts_u64(wa + ((uint32_t)v << 3), (uint64_t)lo | ((uint64_t)hi << 32));
+                // +m at every copy's own step; repeated quarters write the same value to the same place.  Only
+                // for a node with a valid count: then every quarter is a step of the row (1..T); the word of an
+                // absent or overfull node holds no usable positions and the sequence is malformed anyway.
+                if (c >= 1 && c <= limit) {
+                    const MemT mv = __ldg(gm + v);
+                    const uint32_t dm1 = da - (uint32_t)sizeof(MemT);
+                    sts_mem(dm1 + ((lo & 0xFFFFu) << kShift), mv);
+                    sts_mem(dm1 + ((lo >> 16) << kShift), mv);
+                    sts_mem(dm1 + ((hi & 0xFFFFu) << kShift), mv);
+                    sts_mem(dm1 + ((hi >> 16) << kShift), mv);
+                }
             }
             flags = __reduce_or_sync(0xFFFFFFFFu, flags);
             dur = warp_sum64(dur);
