@@ -1050,7 +1050,8 @@ void moc_graph_destroy(moc_graph* g) {
     if (g->h_stage) cudaFreeHost(g->h_stage);
     if (g->copy_stream) {
         cudaStreamDestroy(g->copy_stream);
-        for (cudaEvent_t ev : g->chunk_ev) cudaEventDestroy(ev);
+        for (cudaEvent_t ev : g->chunk_ev)
+            if (ev) cudaEventDestroy(ev);
     }
     for (int li = 0; li < 3; ++li) {
         cudaFree(g->lane[li].d_rec32);

@@ -19,6 +19,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "moc_pair_kernel.cuh"
+
 namespace moc {
 
 constexpr int kEditThreads = 256;   // 8 warps per block, one parent or one edit per warp at a time
@@ -58,6 +60,13 @@ struct PrepParams {
     const int32_t* todo;        // may be null: indices of the parents to (re)build, todo_count of them
     const int32_t* todo_count;  // device counter read by the kernel
     uint32_t warp_bytes;
+    // successor tiles of the warp-per-sequence evaluation kernel (moc_pair_kernel.cuh), read through L1;
+    // n_tiles = 0: not available, the node pass walks the plain successor lists
+    int32_t n_tiles;
+    const void* rec;
+    const uint64_t* wslot;
+    const uint32_t* sell;
+    int64_t base_dur;           // sum of all w
 };
 
 template <typename T>
@@ -101,9 +110,13 @@ __device__ __forceinline__ void edit_add(int64_t* p, int64_t v) {
     atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
 }
 
-// Shared memory of one warp: occurrence words [occ_stride] uint32, then two arrays of stride + 4 MemT.
-__host__ __device__ inline size_t edit_warp_bytes(int32_t occ_stride, int32_t stride, size_t mem_sz) {
-    return (size_t)occ_stride * 4 + 2 * ((((size_t)stride + 4) * mem_sz + 15) & ~size_t(15));
+// Words of the occurrence array of one warp in shared memory: the n nodes, the spare word n, the word n + 1
+// (sequence length, for sinks) and, at the next multiple of four after n + 2, the constant word of empty node slots.
+__host__ __device__ inline int32_t edit_word_stride(int32_t n) { return ((n + 2 + 3) & ~3) + 4; }
+
+// Shared memory of one warp: occurrence words [edit_word_stride(n)] uint32, then two arrays of stride + 4 MemT.
+__host__ __device__ inline size_t edit_warp_bytes(int32_t n, int32_t stride, size_t mem_sz) {
+    return (size_t)edit_word_stride(n) * 4 + 2 * ((((size_t)stride + 4) * mem_sz + 15) & ~size_t(15));
 }
 
 // Full evaluation of every parent (same quantities as the evaluation kernels: Section 2, Eqs. 1-8)
@@ -117,9 +130,9 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
     char* ws = smem + (size_t)warp * p.warp_bytes;
     uint32_t* word = reinterpret_cast<uint32_t*>(ws);
     const size_t arr_bytes = (((size_t)c.stride + 4) * sizeof(MemT) + 15) & ~size_t(15);
-    MemT* arrA = reinterpret_cast<MemT*>(ws + (size_t)c.occ_stride * 4);
-    MemT* arrB = reinterpret_cast<MemT*>(ws + (size_t)c.occ_stride * 4 + arr_bytes);
-    const int32_t n = c.n;
+    const int32_t n = c.n, wstride = edit_word_stride(c.n);
+    MemT* arrA = reinterpret_cast<MemT*>(ws + (size_t)wstride * 4);
+    MemT* arrB = reinterpret_cast<MemT*>(ws + (size_t)wstride * 4 + arr_bytes);
     constexpr uint32_t kFull = 0xFFFFFFFFu;
 
     const int32_t count = p.todo != nullptr ? min(*p.todo_count, c.P) : c.P;
@@ -130,7 +143,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
         int32_t out_st = -2;
         int32_t* row = c.row + (int64_t)b * c.stride;
         if (T >= n && T <= c.max_T) {
-            for (int32_t i = lane; i < c.occ_stride; i += 32) word[i] = 0;
+            for (int32_t i = lane; i < wstride; i += 32) word[i] = 0;
             for (int32_t i = lane; i < c.stride + 4; i += 32) arrA[i] = 0;
             __syncwarp();
             // ---- occurrence words (1-based steps, 16 bits each) and the copy of the row
@@ -149,6 +162,95 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
             bool absent = false, dep = false, over = false;
             int64_t dur = 0;
             int32_t* fre = c.fre + (int64_t)b * c.stride;
+            if (p.n_tiles > 0) {
+                // The node pass of the evaluation kernel: lane l serves the nodes l (mod 32) in tiles of two
+                // slots, successor rows of packed word offsets, two shifted packed reductions per successor
+                // word (end of the last copy with the precedence test, end of the first copy).
+                constexpr uint32_t kRecB = sizeof(MemT) == 4 ? 8u : 16u;
+                const uint32_t wa = (uint32_t)__cvta_generic_to_shared(word);
+                const char* prec = reinterpret_cast<const char*>(p.rec) + kRecB * lane;
+                const uint64_t* pw = p.wslot + lane;
+                const uint32_t* ps = p.sell + lane;
+                uint32_t vmin = 0xFFFFFFFFu, depw = 0, capw = 0;
+                uint64_t acc = 0;
+                const uint32_t empty_off = 4u * (((uint32_t)n + 2u + 3u) & ~3u);   // where the records of empty slots point
+                if (lane == 0) {
+                    word[n + 1] = (uint32_t)T * 0x10001u;               // the made-up successor of sinks
+                    word[empty_off >> 2] = 0x00010001u;
+                }
+                __syncwarp();
+                for (int d = 0; d < p.n_tiles; ++d, prec += 64 * kRecB, pw += 64) {
+                    uint32_t ab[2], naa[2], nbb[2], Ga[2], Gb[2], xoff[2];
+                    MemT mm[2];
+                    int rows = 0;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t x;
+                        if constexpr (sizeof(MemT) == 4) {
+                            const uint2 r = __ldg(reinterpret_cast<const uint2*>(prec + 32 * kRecB * h));
+                            x = r.x;
+                            mm[h] = (MemT)r.y;
+                        } else {
+                            const uint4 r = __ldg(reinterpret_cast<const uint4*>(prec + 32 * kRecB * h));
+                            x = r.x;
+                            mm[h] = (MemT)((uint64_t)r.z | ((uint64_t)r.w << 32));
+                        }
+                        if (h == 0) rows = (int)(x >> 16);
+                        xoff[h] = x & 0xFFFFu;
+                        const uint32_t own = lds_u32(wa + xoff[h]);
+                        vmin = min(vmin, own);
+                        const uint32_t sw = swap_halves(own);
+                        const uint32_t mn = min_u16x2(own, sw), mx = max_u16x2(own, sw);
+                        ab[h] = __byte_perm(mn, mx, 0x7610);
+                        naa[h] = 0x00010000u - mn;
+                        nbb[h] = 0x00010000u - mx;
+                        Ga[h] = mx - mn;
+                        Gb[h] = 0x00010000u - Ga[h];
+                    }
+                    rows = __shfl_sync(kFull, rows, 0);
+                    for (int k = 0; k < rows; ++k, ps += 32) {
+                        const uint32_t e = __ldg(ps);
+                        const uint32_t r0 = lds_u32(wa + (e & 0xFFFFu)), r1 = lds_u32(wa + (e >> 16));
+                        Ga[0] = __viaddmax_u16x2(r0, naa[0], Ga[0]);
+                        Ga[1] = __viaddmax_u16x2(r1, naa[1], Ga[1]);
+                        Gb[0] = __viaddmax_u16x2(r0, nbb[0], Gb[0]);
+                        Gb[1] = __viaddmax_u16x2(r1, nbb[1], Gb[1]);
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        depw |= Ga[h];
+                        const uint32_t gg = max_u16x2(__byte_perm(Ga[h], Gb[h], 0x5410), __byte_perm(Ga[h], Gb[h], 0x7632));
+                        const uint32_t v = gg + ab[h];                   // (end of b, end of a), 1-based
+                        const uint32_t a16 = ab[h] & 0xFFFFu, b16 = ab[h] >> 16, fb = v & 0xFFFFu, fa = v >> 16;
+                        const bool real = xoff[h] != empty_off;          // empty slots own the constant word: no step is theirs
+                        if (real && b16 != 0) {
+                            arrB[b16 - 1] = (MemT)fb - 1;                // free steps gather on chip, written out in order below
+                            edit_add(&arrA[b16 - 1], mm[h]);
+                            edit_add(&arrA[fb], (MemT)(-mm[h]));
+                            if (a16 != b16) {
+                                arrB[a16 - 1] = (MemT)fa - 1;
+                                edit_add(&arrA[a16 - 1], mm[h]);
+                                edit_add(&arrA[fa], (MemT)(-mm[h]));
+                                const uint64_t wx = __ldg(pw + 32 * h);
+                                capw |= (uint32_t)(wx >> 32);
+                                acc += wx;
+                            }
+                        }
+                    }
+                }
+                vmin = __reduce_min_sync(kFull, vmin);
+                int64_t accs = (int64_t)acc;
+                for (int dd = 16; dd > 0; dd >>= 1) accs += __shfl_xor_sync(kFull, accs, dd);
+                const uint64_t acc_all = (uint64_t)accs;
+                absent = vmin == 0;
+                over = __any_sync(kFull, (int32_t)capw < 0) || (int)((acc_all >> kPairCntShift) & 0x7FFFu) != T - n;
+                dep = (depw & 0x80008000u) != 0;
+                __syncwarp();
+                for (int32_t t = lane; t < T; t += 32) fre[t] = (int32_t)arrB[t];
+                // position sum and duration in the form the rest of the kernel expects
+                vsum = lane == 0 ? (uint32_t)T * ((uint32_t)T + 1u) / 2u : 0u;
+                dur = lane == 0 ? p.base_dur + (int64_t)(acc_all & kPairDurMask) : 0;
+            } else
             for (int32_t u = lane; u < n; u += 32) {
                 const uint32_t wd = word[u];
                 const uint32_t lo = wd & 0xFFFFu, hi = wd >> 16;
@@ -191,7 +293,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                 out_du = dur;
             } else if (well) {
                 // ---- profile, prefix maxima, suffix maxima: lane owns a run of consecutive steps
-                const int32_t per = (T + 31) / 32;
+                const int32_t per = ((T + 31) / 32) | 1;                  // odd: the lanes' runs start in different banks
                 const int32_t t0 = min(T, lane * per), t1 = min(T, t0 + per);
                 MemT sum = 0;
                 for (int32_t t = t0; t < t1; ++t) sum += arrA[t];

@@ -33,6 +33,14 @@ int cache_prepare(moc_cache* h, const int32_t* seqs, const int32_t* lens, const 
     p.todo = todo;
     p.todo_count = todo_count;
     p.warp_bytes = (uint32_t)h->warp_bytes;
+    // the successor tiles of the warp-per-sequence kernel, when the graph has them and its durations fit their packing
+    const moc_graph* g = h->g;
+    const bool tiles = g->d_rec32 != nullptr && g->C <= 2 && (__int128)g->C * g->sum_w < ((__int128)1 << 48);
+    p.n_tiles = tiles ? g->n_tiles : 0;
+    p.rec = h->wide ? g->d_rec64 : g->d_rec32;
+    p.wslot = g->d_wslot;
+    p.sell = g->d_sell;
+    p.base_dur = g->sum_w;
     auto fn = h->wide ? moc::edit_prepare_kernel<int64_t> : moc::edit_prepare_kernel<int32_t>;
     MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
     const int grid = (int)std::min<int64_t>(h->grid_cap, ((int64_t)P + h->wpb - 1) / h->wpb);
@@ -61,7 +69,7 @@ int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
     h->wide = g->sum_m > (int64_t)INT32_MAX / g->C;
     const size_t msz = h->wide ? 8 : 4;
     const int32_t stride = (int32_t)((max_T + 3) & ~int64_t(3)), occ_stride = (g->n + 1 + 3) & ~3;
-    h->warp_bytes = moc::edit_warp_bytes(occ_stride, stride, msz);
+    h->warp_bytes = moc::edit_warp_bytes(g->n, stride, msz);
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
     if (h->warp_bytes > cap) {
         delete h;
