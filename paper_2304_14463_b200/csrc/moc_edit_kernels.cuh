@@ -148,13 +148,20 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
             __syncwarp();
             // ---- occurrence words (1-based steps, 16 bits each) and the copy of the row
             const int32_t* src = p.seqs + p.offs[b];
-            for (int32_t t = lane; t < T; t += 32) {
-                const int32_t v = __ldg(src + t);
+            auto put = [&](int32_t v, int32_t t) {
                 row[t] = v;
                 const uint32_t slot = min((uint32_t)v, (uint32_t)n);      // ids outside [0, n) land in a spare word
                 const uint32_t t1 = (uint32_t)t + 1u;
                 const uint32_t old = atomicExch(&word[slot], t1 * 0x10001u);
                 if (old) reinterpret_cast<uint16_t*>(&word[slot])[1] = (uint16_t)old;
+            };
+            for (int32_t t0 = lane; t0 < T; t0 += 256) {                  // eight loads in flight per lane
+                int32_t v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[k] = t0 + 32 * k < T ? __ldg(src + t0 + 32 * k) : 0;
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (t0 + 32 * k < T) put(v[k], t0 + 32 * k);
             }
             __syncwarp();
             // ---- per node: both copies a <= b, free steps from the successors' copies, profile deltas
@@ -208,8 +215,10 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                         Gb[h] = 0x00010000u - Ga[h];
                     }
                     rows = __shfl_sync(kFull, rows, 0);
+                    uint32_t e_next = rows > 0 ? __ldg(ps) : 0u;           // one row ahead: the tiles come through L1
                     for (int k = 0; k < rows; ++k, ps += 32) {
-                        const uint32_t e = __ldg(ps);
+                        const uint32_t e = e_next;
+                        if (k + 1 < rows) e_next = __ldg(ps + 32);
                         const uint32_t r0 = lds_u32(wa + (e & 0xFFFFu)), r1 = lds_u32(wa + (e >> 16));
                         Ga[0] = __viaddmax_u16x2(r0, naa[0], Ga[0]);
                         Ga[1] = __viaddmax_u16x2(r1, naa[1], Ga[1]);
