@@ -357,14 +357,27 @@ int moc_search_set_kinds(moc_search* s, uint32_t kinds);
  *                proposal with the smallest key among those with status >= 0, the lowest e among
  *                equals, and it replaces the chain's sequence when its key is not larger.  E = 1 is
  *                the single proposal described above.
- *   incremental  0: every proposal is written out and evaluated from scratch (E must be 1);
- *                1: proposals are scored from the cached evaluation of the chain's sequence
- *                (moc_eval_edits) and only accepted ones are written out.  Needs C <= 2 and a valid
- *                sequence (status >= 0) in every chain at the time of the call (MOC_ERR_ARG otherwise).
- *                The two ways give identical chains.
+ *   incremental  0 (MOC_SEARCH_WRITTEN_OUT): every proposal is written out and evaluated from scratch
+ *                (E must be 1);
+ *                1 (MOC_SEARCH_SCORE_AUTO): proposals are scored from the cached evaluation of the chain's
+ *                sequence and only accepted ones are written out; the library picks the scoring kernel
+ *                (a warp per chain from E = 4 on when the graph fits it, else a warp per proposal);
+ *                2 (MOC_SEARCH_SCORE_EDIT): the same with a warp per proposal: a generation is four
+ *                kernels (draw, moc_eval_edits, pick, rebuild of the changed cache entries);
+ *                3 (MOC_SEARCH_SCORE_CHAIN): the same with a warp per chain: the chain's cache entry is
+ *                staged in shared memory once and its E proposals are drawn, scored and settled there;
+ *                a generation is two kernels (that one and the rebuild).  MOC_ERR_ARG when the entry
+ *                and the correction lists (4 + 2 * largest in-degree entries) of four chains do not
+ *                fit the shared memory of an SM.
+ *                1 to 3 need C <= 2 and a valid sequence (status >= 0) in every chain at the time of
+ *                the call (MOC_ERR_ARG otherwise).  All four give identical chains.
  * Synchronises the device, allocates (the cache of the chains, 28 bytes per proposal); after it
- * moc_search_run allocates nothing.  With incremental = 1 a generation is four kernels.
+ * moc_search_run allocates nothing.
  */
+#define MOC_SEARCH_WRITTEN_OUT 0
+#define MOC_SEARCH_SCORE_AUTO 1
+#define MOC_SEARCH_SCORE_EDIT 2
+#define MOC_SEARCH_SCORE_CHAIN 3
 int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental);
 
 /*

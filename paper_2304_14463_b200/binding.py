@@ -454,8 +454,10 @@ class Search:
         moc_search_set_kinds(self.h, kinds)
 
     def set_samples(self, samples, incremental=True):
-        """samples proposals per chain and generation; incremental: scored from the cached evaluation."""
-        _check(lib.moc_search_set_samples(self.h, int(samples), 1 if incremental else 0), "moc_search_set_samples")
+        """samples proposals per chain and generation; incremental: False / 0 written out and evaluated from
+        scratch, True / 1 scored from the cached evaluation (the library picks the kernel), 2 with a warp per
+        proposal, 3 with a warp per chain (MOC_SEARCH_*)."""
+        _check(lib.moc_search_set_samples(self.h, int(samples), int(incremental)), "moc_search_set_samples")
 
     def info(self):
         return moc_search_info(self.h)
@@ -474,6 +476,7 @@ class Search:
 
 
 MOC_STATUS_PARENT_INVALID = -3
+MOC_SEARCH_WRITTEN_OUT, MOC_SEARCH_SCORE_AUTO, MOC_SEARCH_SCORE_EDIT, MOC_SEARCH_SCORE_CHAIN = 0, 1, 2, 3
 
 
 class EditCache:

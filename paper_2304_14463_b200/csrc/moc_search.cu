@@ -8,6 +8,7 @@
 
 #include "moc_cache_host.cuh"
 #include "moc_search_kernels.cuh"
+#include "moc_search_score_kernel.cuh"
 
 using namespace moc_host;
 
@@ -27,6 +28,10 @@ struct moc_search {
     moc_cache* cache = nullptr;
     char* d_inc = nullptr;
     moc::SearchIncParams ip{};
+    // one kernel per generation with a warp per chain (moc_search_score_kernel.cuh) instead of draw, score, pick
+    bool fused = false;
+    moc::ScoreParams sp{};
+    int score_wpb = 0, score_grid_cap = 0;
 };
 
 namespace {
@@ -34,6 +39,40 @@ namespace {
 size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 
 int chain_blocks(int32_t P) { return (P + moc::kSearchThreads / 32 - 1) / (moc::kSearchThreads / 32); }
+
+// Launch shape of the warp-per-chain generation kernel; false when the graph's largest in-degree or the row
+// length leaves fewer than four warps on an SM.
+bool plan_fused(moc_search* s) {
+    const moc_graph* g = s->g;
+    const moc_cache* h = s->cache;
+    moc::ScoreParams& sp = s->sp;
+    const size_t msz = h->wide ? 8 : 4;
+    const int32_t worst = 4 + 2 * g->max_indeg;
+    sp.list_cap = std::max(192, (worst + 31) & ~31);
+    sp.warp_bytes = (uint32_t)moc::score_warp_bytes(h->c.occ_stride, h->c.stride, msz, sp.list_cap, &sp.fre_b, &sp.prof_b,
+                                                   &sp.lh_b, &sp.val_b);
+    const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
+    if ((size_t)sp.warp_bytes * 4 > cap) return false;
+    auto fn = h->wide ? moc::search_score_kernel<int64_t> : moc::search_score_kernel<int32_t>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(g->smem_optin - 1024)) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    int best = 0;
+    for (int k = 1; k <= moc::kScoreThreads / 32; ++k) {
+        const size_t blk = (size_t)sp.warp_bytes * k;
+        if (blk > cap) break;
+        int nb = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, 32 * k, blk) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        if (nb * k > best) { best = nb * k; s->score_wpb = k; }
+    }
+    if (best < 4) return false;
+    s->score_grid_cap = g->sm_count * (best / s->score_wpb);
+    return true;
+}
 
 }  // namespace
 
@@ -138,6 +177,29 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
     moc::SearchParams& p = s->p;
     const int blocks = chain_blocks(s->P);
     int launches = 0;
+    if (s->incremental && s->fused) {
+        moc_cache* h = s->cache;
+        if (h->graph_generation != h->g->generation)
+            return fail(MOC_ERR_ARG, "moc_search_run: the graph's C or node caps changed after the search's cache was built");
+        auto fn = h->wide ? moc::search_score_kernel<int64_t> : moc::search_score_kernel<int32_t>;
+        const int wpb = s->score_wpb;
+        const int grid = (int)std::min<int64_t>(s->score_grid_cap, ((int64_t)s->P + wpb - 1) / wpb);
+        for (int32_t k = 0; k < n_generations; ++k) {
+            p.generation = s->generation + (uint32_t)k;
+            s->sp.s = p;
+            s->sp.c = h->c;
+            s->sp.c.cap = h->g->d_cap;
+            fn<<<grid, 32 * wpb, (size_t)s->sp.warp_bytes * wpb, st>>>(s->sp);
+            int rc = cache_prepare(h, p.rows, p.lens, s->ip.row_offs, s->P, s->ip.todo, s->ip.todo_count + (p.generation & 1u),
+                                   s->M, nullptr, nullptr, nullptr, st);
+            if (rc != MOC_OK) return rc;
+            launches += 2;
+        }
+        MOC_CUDA(cudaGetLastError());
+        s->generation += (uint32_t)n_generations;
+        launch_counter() = launches;
+        return MOC_OK;
+    }
     if (s->incremental) {
         const int64_t nE = (int64_t)s->P * s->samples;
         for (int32_t k = 0; k < n_generations; ++k) {
@@ -186,8 +248,8 @@ int moc_search_set_kinds(moc_search* s, uint32_t kinds) {
 
 int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) {
     clear_error();
-    if (!s || samples < 1 || samples > 4096 || (incremental != 0 && incremental != 1))
-        return fail(MOC_ERR_ARG, "moc_search_set_samples: null handle, samples outside [1, 4096] or flag outside {0, 1}");
+    if (!s || samples < 1 || samples > 4096 || incremental < 0 || incremental > 3)
+        return fail(MOC_ERR_ARG, "moc_search_set_samples: null handle, samples outside [1, 4096] or mode outside 0..3");
     if (samples > 1 && !incremental)
         return fail(MOC_ERR_ARG, "moc_search_set_samples: more than one proposal per chain needs the incremental evaluation");
     if ((int64_t)s->P * samples > INT32_MAX) return fail(MOC_ERR_ARG, "moc_search_set_samples: P * samples exceeds 2^31 - 1");
@@ -196,6 +258,7 @@ int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) 
     MOC_CUDA(cudaDeviceSynchronize());          // generations in flight still use the old buffers
     if (!incremental) {
         s->incremental = false;
+        s->fused = false;
         s->samples = 1;
         return MOC_OK;
     }
@@ -216,7 +279,7 @@ int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) 
     const size_t o_par = 0, o_op = o_par + up256(nE * 4), o_q = o_op + up256(nE * 4), o_j = o_q + up256(nE * 4),
                  o_st = o_j + up256(nE * 4), o_pk = o_st + up256(nE * 4), o_du = o_pk + up256(nE * 8),
                  o_offs = o_du + up256(nE * 8), o_todo = o_offs + up256((bP + 1) * 8), o_cnt = o_todo + up256(bP * 4),
-                 total = o_cnt + 256;
+                 total = o_cnt + 256;          // o_cnt: two counters, used in turn by the warp-per-chain kernel
     if (s->d_inc) MOC_CUDA(cudaFree(s->d_inc));
     s->d_inc = nullptr;
     s->incremental = false;
@@ -239,6 +302,22 @@ int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) 
     ip.row_offs = (int64_t*)(b + o_offs);
     ip.todo = (int32_t*)(b + o_todo);
     ip.todo_count = (int32_t*)(b + o_cnt);
+    MOC_CUDA(cudaMemset(ip.todo_count, 0, 8));
+    // scoring kernel: a warp per chain when asked for, or by default from four proposals per chain on
+    s->fused = false;
+    if (incremental == MOC_SEARCH_SCORE_CHAIN || (incremental == MOC_SEARCH_SCORE_AUTO && samples >= 4)) {
+        s->fused = plan_fused(s);
+        if (!s->fused && incremental == MOC_SEARCH_SCORE_CHAIN) {
+            cudaFree(s->d_inc);
+            s->d_inc = nullptr;
+            return fail(MOC_ERR_ARG, "moc_search_set_samples: the warp-per-chain kernel cannot hold this graph's rows and "
+                        "correction lists (n = %d, largest in-degree %d) in shared memory", s->g->n, s->g->max_indeg);
+        }
+    }
+    s->sp.samples = samples;
+    s->sp.row_offs = ip.row_offs;
+    s->sp.todo = ip.todo;
+    s->sp.todo_count = ip.todo_count;
     // cache of all chains from their current rows
     moc::search_row_offsets_kernel<<<(s->P + 255) / 256, 256>>>(ip);
     int rc = cache_prepare(s->cache, s->p.rows, s->p.lens, ip.row_offs, s->P, nullptr, nullptr, s->M, nullptr, nullptr, nullptr, nullptr);
