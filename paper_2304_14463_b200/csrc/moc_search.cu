@@ -50,7 +50,7 @@ bool plan_fused(moc_search* s) {
     const int32_t worst = 4 + 2 * g->max_indeg;
     sp.list_cap = std::max(192, (worst + 31) & ~31);
     sp.warp_bytes = (uint32_t)moc::score_warp_bytes(h->c.occ_stride, h->c.stride, msz, sp.list_cap, &sp.fre_b, &sp.prof_b,
-                                                   &sp.lh_b, &sp.val_b);
+                                                   &sp.lh_b, &sp.val_b, &sp.diff_b);
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
     if ((size_t)sp.warp_bytes * 4 > cap) return false;
     auto fn = h->wide ? moc::search_score_kernel<int64_t> : moc::search_score_kernel<int32_t>;

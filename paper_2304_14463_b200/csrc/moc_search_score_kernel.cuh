@@ -11,7 +11,8 @@
 // range corrections to the parent's profile (one entry per retention interval that changes: at most
 // 4 for the edited node and 2 for each of its predecessors).  The one part that is long, the maximum
 // of the corrected profile over the recomputed window, runs with the whole warp on one proposal at a
-// time: lane i takes the window steps i, i + 32, ... and adds the corrections that cover its step.
+// time: the corrections go into a difference array, each lane takes a run of consecutive window steps,
+// and a warp scan carries the running correction from run to run.
 // Only proposals that passed both tests (about a fifth of random ones) reach that part.
 //
 // The correction lists of the lanes share `list_cap` entries of shared memory.  When the admissible
@@ -33,13 +34,15 @@ struct ScoreParams {
     int32_t* todo;          // P: chains whose sequence changed in this generation
     int32_t* todo_count;    // two counters: [generation & 1] collects this generation's chains, the other is cleared
     uint32_t warp_bytes;    // shared memory of one warp
-    uint32_t fre_b, prof_b, lh_b, val_b;   // byte offsets of its parts (copy positions come first)
+    uint32_t fre_b, prof_b, lh_b, val_b, diff_b;   // byte offsets of its parts (copy positions come first)
     int32_t list_cap;
 };
 
-// Bytes of one warp: copy positions (occ_stride words), free steps (16 bits each), profile, range list.
+// Bytes of one warp: copy positions (occ_stride words), free steps (16 bits each), profile, range list,
+// difference array of the corrections (stride + 4 entries).
 __host__ __device__ inline size_t score_warp_bytes(int32_t occ_stride, int32_t stride, size_t mem_sz, int32_t list_cap,
-                                                   uint32_t* fre_b, uint32_t* prof_b, uint32_t* lh_b, uint32_t* val_b) {
+                                                   uint32_t* fre_b, uint32_t* prof_b, uint32_t* lh_b, uint32_t* val_b,
+                                                   uint32_t* diff_b) {
     size_t o = (size_t)occ_stride * 4;
     *fre_b = (uint32_t)o;
     o += ((size_t)stride * 2 + 15) & ~size_t(15);
@@ -49,6 +52,8 @@ __host__ __device__ inline size_t score_warp_bytes(int32_t occ_stride, int32_t s
     o += ((size_t)list_cap * mem_sz + 15) & ~size_t(15);
     *lh_b = (uint32_t)o;
     o += ((size_t)list_cap * 4 + 15) & ~size_t(15);
+    *diff_b = (uint32_t)o;
+    o += (((size_t)stride + 4) * mem_sz + 15) & ~size_t(15);
     return o;
 }
 
@@ -65,6 +70,8 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
     MemT* prof = reinterpret_cast<MemT*>(mine + p.prof_b);
     MemT* rv = reinterpret_cast<MemT*>(mine + p.val_b);
     uint32_t* rl = reinterpret_cast<uint32_t*>(mine + p.lh_b);
+    MemT* diff = reinterpret_cast<MemT*>(mine + p.diff_b);
+    for (int32_t i = lane; i < c.stride + 4; i += 32) diff[i] = 0;
     constexpr uint32_t kFull = 0xFFFFFFFFu;
     constexpr int64_t kInf = INT64_MAX;
     if (blockIdx.x == 0 && threadIdx.x == 0) p.todo_count[(s.generation + 1u) & 1u] = 0;
@@ -274,19 +281,33 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                     const int32_t ji_s = __shfl_sync(kFull, ji, sl), qd_s = __shfl_sync(kFull, qd, sl);
                     const int32_t lb = __shfl_sync(kFull, lbase, sl), lc = __shfl_sync(kFull, lcnt, sl);
                     const MemT cr_s = __shfl_sync(kFull, cross, sl);
+                    // corrections as a difference array over the child steps (zero outside this block of code)
+                    for (int32_t k = lane; k < lc; k += 32) {
+                        const uint32_t lh = rl[lb + k];
+                        const MemT v = rv[lb + k];
+                        edit_add(&diff[lh & 0xFFFFu], v);
+                        edit_add(&diff[lh >> 16], (MemT)(-v));
+                    }
+                    __syncwarp();
+                    // lane owns a run of consecutive window steps (odd length: the runs start in different banks)
+                    const int32_t L = hi - lo + 1;
+                    const int32_t per = ((L + 31) / 32) | 1;
+                    const int32_t t0 = lo + min(L, lane * per), t1 = lo + min(L, (lane + 1) * per);
+                    MemT sum = 0;
+                    for (int32_t t = t0; t < t1; ++t) sum += diff[t];
+                    MemT run = edit_warp_incl_sum(sum, lane) - sum;
                     MemT top = 0;
-                    for (int32_t t = lo + lane; t <= hi; t += 32) {
-                        const int32_t t1 = t - (t > ji_s ? 1 : 0);
-                        MemT u = t == ji_s ? cr_s : prof[t1 + (t1 >= qd_s ? 1 : 0)];
-                        for (int32_t k = 0; k < lc; ++k) {
-                            const uint32_t lh = rl[lb + k];
-                            const MemT v = rv[lb + k];
-                            if ((uint32_t)t >= (lh & 0xFFFFu) && (uint32_t)t < (lh >> 16)) u += v;
-                        }
+                    for (int32_t t = t0; t < t1; ++t) {
+                        run += diff[t];
+                        diff[t] = 0;
+                        const int32_t tt = t - (t > ji_s ? 1 : 0);
+                        const MemT u = run + (t == ji_s ? cr_s : prof[tt + (tt >= qd_s ? 1 : 0)]);
                         top = u > top ? u : top;
                     }
+                    if (lane == 0) diff[hi + 1] = 0;
                     top = edit_warp_max(top);
                     if (lane == sl) best = top > best ? top : best;
+                    __syncwarp();
                 }
                 if (act) {
                     out_pk = (int64_t)best;
