@@ -198,6 +198,110 @@ def test_search_incremental_parity(B, idx, P, samples):
         assert_state_equal(S, OS, "after switching back")
 
 
+def _run_scored(B, n, edges, w, m, C, seqs, lens, M, samples, mode, gens, caps=None, kinds=7, what=""):
+    G = B.Graph(n, edges, w, m, C)
+    O = OracleGraph(n, edges, w, m, C)
+    if caps is not None:
+        G.set_caps(caps)
+        O.set_caps(caps)
+    S = B.Search(G, dev(seqs), dev(lens), M, 23)
+    if kinds != 7:
+        S.set_kinds(kinds)
+    S.set_samples(samples, incremental=mode)
+    OS = OracleSearch(O, seqs, lens, M, 23, stride=S.info()["stride"], kinds=kinds, samples=samples)
+    for g in gens:
+        S.run(g)
+        OS.run(g)
+        assert_state_equal(S, OS, f"{what}: mode {mode}, {samples} samples, after {OS.generation}")
+    return S, OS
+
+
+@pytest.mark.parametrize("mode", [2, 3])
+@pytest.mark.parametrize("idx,P,samples", [(0, 256, 5), (1, 128, 33), (2, 96, 16), (2, 48, 70)])
+def test_search_scoring_kernels_agree_with_oracle(B, idx, P, samples, mode):
+    """The two scoring kernels of the search on the cached evaluation, each forced: a warp per proposal (2) and
+    a warp per chain (3; fewer proposals than lanes, a pass and a bit, more than two passes)."""
+    wl = W.make(idx, seed=4, B=P)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    S, OS = _run_scored(B, wl.n, wl.edges, wl.w, wl.m, wl.C, wl.seqs, wl.lens, M, samples, mode, (1, 3, 20), what=f"config {idx}")
+    assert OS.accepted > 0
+    # the other kernel takes over the same chains in mid-search
+    S.set_samples(samples, incremental=5 - mode)
+    S.run(5)
+    OS.run(5)
+    assert_state_equal(S, OS, "after switching the scoring kernel")
+
+
+@pytest.mark.parametrize("mode", [2, 3])
+def test_search_scoring_caps_kinds_and_wide(B, mode):
+    """Per-node caps, restricted kinds of edit and 64-bit memory sums through both scoring kernels."""
+    wl = W.make(1, seed=6, B=96)
+    rng = np.random.default_rng(11)
+    caps = np.where(rng.random(wl.n) < 0.5, 1, 2).astype(np.int32)
+    rows = [np.arange(wl.n, dtype=np.int32) for _ in range(96)]           # the identity order respects every cap
+    seqs, lens = W.pack(rows)
+    O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
+    M = O0.eval(np.arange(wl.n), 1 << 60)["peak"] * 80 // 100
+    _, OS = _run_scored(B, wl.n, wl.edges, wl.w, wl.m, wl.C, seqs, lens, M, 12, mode, (2, 30), caps=caps, what="caps")
+    assert OS.accepted > 0
+    for kinds in (1, 3, 6):
+        _run_scored(B, wl.n, wl.edges, wl.w, wl.m, wl.C, wl.seqs, wl.lens, M, 9, mode, (1, 12), kinds=kinds, what=f"kinds {kinds}")
+    big = wl.m * (1 << 33)
+    _, OS = _run_scored(B, wl.n, wl.edges, wl.w, big, wl.C, wl.seqs, wl.lens, M * (1 << 33), 40, mode, (1, 15), what="wide")
+    assert OS.accepted > 0 and int(OS.peak.max()) > (1 << 40)
+
+
+def _layered_dense(width, layers, seed):
+    """Every node of a layer feeds every node of the next: in-degree = out-degree = width."""
+    rng = np.random.default_rng(seed)
+    n = width * layers
+    edges = np.array([(a * width + i, (a + 1) * width + k) for a in range(layers - 1) for i in range(width)
+                      for k in range(width)], np.int32)
+    return n, edges, rng.integers(1, 50, n).astype(np.int64), rng.integers(1, 1000, n).astype(np.int64)
+
+
+def test_search_chain_kernel_in_rounds(B):
+    """In-degree 30: one proposal may need 64 entries of the 192-entry correction list of a warp, so a pass with
+    more than three admissible proposals is scored in several rounds.  A copy inserted behind the node's first one
+    is always admissible, so with inserts only about half of the 32 proposals of a pass are."""
+    n, edges, w, m = _layered_dense(30, 3, 2)
+    rng = np.random.default_rng(3)
+    rows = []
+    for _ in range(48):
+        r = np.concatenate([rng.permutation(30) + 30 * a for a in range(3)]).astype(np.int32)
+        rows.append(r)
+    seqs, lens = W.pack(rows)
+    O0 = OracleGraph(n, edges, w, m, 2)
+    M = O0.eval(np.arange(n), 1 << 60)["peak"] * 90 // 100
+    for mode in (3, 2):
+        _run_scored(B, n, edges, w, m, 2, seqs, lens, M, 32, mode, (1, 2, 10), kinds=1, what="dense, inserts")
+        _, OS = _run_scored(B, n, edges, w, m, 2, seqs, lens, M, 48, mode, (1, 8), what="dense, all kinds")
+        assert OS.accepted > 0
+
+
+def test_search_chain_kernel_refuses_what_it_cannot_hold(B):
+    """A graph whose rows and correction lists do not fit four warps of an SM: the warp-per-chain kernel is
+    refused when asked for by name, and the automatic choice scores with a warp per proposal instead."""
+    n = 1700
+    edges = np.array([(i, n - 1) for i in range(n - 1)], np.int32)          # in-degree 1699
+    rng = np.random.default_rng(1)
+    w, m = rng.integers(1, 9, n).astype(np.int64), rng.integers(1, 99, n).astype(np.int64)
+    rows = [np.concatenate([rng.permutation(n - 1), [n - 1]]).astype(np.int32) for _ in range(6)]
+    seqs, lens = W.pack(rows)
+    G = B.Graph(n, edges, w, m, 2)
+    S = B.Search(G, dev(seqs), dev(lens), 1 << 60, 5)
+    with pytest.raises(B.MocError) as e:
+        S.set_samples(8, incremental=3)
+    assert e.value.code == -1 and "in-degree" in str(e.value)
+    O = OracleGraph(n, edges, w, m, 2)
+    S.set_samples(8, incremental=1)
+    OS = OracleSearch(O, seqs, lens, 1 << 60, 5, stride=S.info()["stride"], samples=8)
+    S.run(3)
+    OS.run(3)
+    assert_state_equal(S, OS, "star graph, automatic choice")
+
+
 def test_search_incremental_errors(B):
     wl = W.make(1, seed=3, B=32)
     O0 = OracleGraph(wl.n, wl.edges, wl.w, wl.m, wl.C)
@@ -213,6 +317,8 @@ def test_search_incremental_errors(B):
         S.set_samples(4, incremental=False)                 # several samples need the incremental evaluation
     with pytest.raises(B.MocError):
         S.set_samples(0, incremental=True)
+    with pytest.raises(B.MocError):
+        S.set_samples(4, incremental=4)                     # modes are 0..3
     S.run(3)                                                # still usable in the old way
     wl3 = W.make(3, seed=1, B=8)                            # C = 3: outside the incremental evaluation
     G3 = B.Graph(wl3.n, wl3.edges, wl3.w, wl3.m, wl3.C)
