@@ -32,6 +32,8 @@ struct moc_search {
     bool fused = false;
     moc::ScoreParams sp{};
     int score_wpb = 0, score_grid_cap = 0;
+    const void* score_fn = nullptr;
+    size_t score_smem = 0;
 };
 
 namespace {
@@ -53,21 +55,32 @@ bool plan_fused(moc_search* s) {
                                                    &sp.lh_b, &sp.val_b, &sp.diff_b);
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
     if ((size_t)sp.warp_bytes * 4 > cap) return false;
-    auto fn = h->wide ? moc::search_score_kernel<int64_t> : moc::search_score_kernel<int32_t>;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(g->smem_optin - 1024)) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
+    // with the block's own copy of the graph when that still leaves eight warps on an SM, else from global memory
+    const int64_t E = g->n_edges;
+    sp.graph_bytes = (uint32_t)moc::score_graph_bytes(g->n, E, msz, &sp.gs_pred_b, &sp.gs_m_b, &sp.gs_succ_b, &sp.gs_predl_b);
     int best = 0;
-    for (int k = 1; k <= moc::kScoreThreads / 32; ++k) {
-        const size_t blk = (size_t)sp.warp_bytes * k;
-        if (blk > cap) break;
-        int nb = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, 32 * k, blk) != cudaSuccess) {
+    for (int chip = 1; chip >= 0; --chip) {
+        if (chip && (g->n > 65535 || sp.graph_bytes > cap / 4)) continue;
+        s->score_fn = chip ? (h->wide ? (const void*)moc::search_score_kernel<int64_t, true> : (const void*)moc::search_score_kernel<int32_t, true>)
+                           : (h->wide ? (const void*)moc::search_score_kernel<int64_t, false> : (const void*)moc::search_score_kernel<int32_t, false>);
+        if (cudaFuncSetAttribute(s->score_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(g->smem_optin - 1024)) != cudaSuccess) {
             cudaGetLastError();
             return false;
         }
-        if (nb * k > best) { best = nb * k; s->score_wpb = k; }
+        const size_t fixed = chip ? sp.graph_bytes : 0;
+        best = 0;
+        for (int k = 1; k <= moc::kScoreThreads / 32; ++k) {
+            const size_t blk = fixed + (size_t)sp.warp_bytes * k;
+            if (blk > cap) break;
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, s->score_fn, 32 * k, blk) != cudaSuccess) {
+                cudaGetLastError();
+                return false;
+            }
+            if (nb * k >= best && nb > 0) { best = nb * k; s->score_wpb = k; }     // ties: the larger block (one copy of the graph)
+        }
+        s->score_smem = fixed + (size_t)sp.warp_bytes * s->score_wpb;
+        if (best >= 8) break;
     }
     if (best < 4) return false;
     s->score_grid_cap = g->sm_count * (best / s->score_wpb);
@@ -181,7 +194,6 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
         moc_cache* h = s->cache;
         if (h->graph_generation != h->g->generation)
             return fail(MOC_ERR_ARG, "moc_search_run: the graph's C or node caps changed after the search's cache was built");
-        auto fn = h->wide ? moc::search_score_kernel<int64_t> : moc::search_score_kernel<int32_t>;
         const int wpb = s->score_wpb;
         const int grid = (int)std::min<int64_t>(s->score_grid_cap, ((int64_t)s->P + wpb - 1) / wpb);
         for (int32_t k = 0; k < n_generations; ++k) {
@@ -189,7 +201,8 @@ int moc_search_run(moc_search* s, int32_t n_generations, void* stream) {
             s->sp.s = p;
             s->sp.c = h->c;
             s->sp.c.cap = h->g->d_cap;
-            fn<<<grid, 32 * wpb, (size_t)s->sp.warp_bytes * wpb, st>>>(s->sp);
+            void* args[] = {&s->sp};
+            MOC_CUDA(cudaLaunchKernel(s->score_fn, dim3(grid), dim3(32 * wpb), args, s->score_smem, st));
             int rc = cache_prepare(h, p.rows, p.lens, s->ip.row_offs, s->P, s->ip.todo, s->ip.todo_count + (p.generation & 1u),
                                    s->M, nullptr, nullptr, nullptr, st);
             if (rc != MOC_OK) return rc;

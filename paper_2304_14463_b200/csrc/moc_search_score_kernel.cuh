@@ -24,7 +24,7 @@
 
 namespace moc {
 
-constexpr int kScoreThreads = 256;
+constexpr int kScoreThreads = 512;
 
 struct ScoreParams {
     SearchParams s;
@@ -33,6 +33,8 @@ struct ScoreParams {
     int64_t* row_offs;      // P + 1: offset of every chain's current row (input of the cache rebuild)
     int32_t* todo;          // P: chains whose sequence changed in this generation
     int32_t* todo_count;    // two counters: [generation & 1] collects this generation's chains, the other is cleared
+    uint32_t graph_bytes;   // shared memory of the block's copy of the graph (kGraphOnChip), a multiple of 16
+    uint32_t gs_pred_b, gs_m_b, gs_succ_b, gs_predl_b;   // its parts after the successor offsets
     uint32_t warp_bytes;    // shared memory of one warp
     uint32_t fre_b, prof_b, lh_b, val_b, diff_b;   // byte offsets of its parts (copy positions come first)
     int32_t list_cap;
@@ -57,14 +59,55 @@ __host__ __device__ inline size_t score_warp_bytes(int32_t occ_stride, int32_t s
     return o;
 }
 
-template <typename MemT>
-__global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const ScoreParams p) {
+// Bytes of the block's copy of the graph: successor and predecessor offsets (n + 1 words each), output sizes
+// (n MemT), successor and predecessor lists (16 bits per entry).
+__host__ __device__ inline size_t score_graph_bytes(int32_t n, int64_t n_edges, size_t mem_sz, uint32_t* pred_b, uint32_t* m_b,
+                                                    uint32_t* succ_b, uint32_t* predl_b) {
+    size_t o = ((size_t)(n + 1) * 4 + 15) & ~size_t(15);
+    *pred_b = (uint32_t)o;
+    o += ((size_t)(n + 1) * 4 + 15) & ~size_t(15);
+    *m_b = (uint32_t)o;
+    o += ((size_t)n * mem_sz + 15) & ~size_t(15);
+    *succ_b = (uint32_t)o;
+    o += ((size_t)n_edges * 2 + 15) & ~size_t(15);
+    *predl_b = (uint32_t)o;
+    o += ((size_t)n_edges * 2 + 15) & ~size_t(15);
+    return o;
+}
+
+// kGraphOnChip: the block keeps the graph's lists and output sizes in shared memory (every lane walks them
+// at its own node, and what the warps' arrays leave of the L1 is too small to hold them).
+template <typename MemT, bool kGraphOnChip>
+__global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const ScoreParams p) {
     extern __shared__ __align__(16) char smem[];
     const EditCacheDev& c = p.c;
     const SearchParams& s = p.s;
     const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
-    char* mine = smem + (size_t)warp * p.warp_bytes;
+    const uint32_t* s_succ_start = reinterpret_cast<const uint32_t*>(smem);
+    const uint32_t* s_pred_start = reinterpret_cast<const uint32_t*>(smem + p.gs_pred_b);
+    const MemT* s_m = reinterpret_cast<const MemT*>(smem + p.gs_m_b);
+    const uint16_t* s_succ = reinterpret_cast<const uint16_t*>(smem + p.gs_succ_b);
+    const uint16_t* s_pred = reinterpret_cast<const uint16_t*>(smem + p.gs_predl_b);
+    if (kGraphOnChip) {
+        const int32_t E = __ldg(&c.succ_start[c.n]);
+        for (int32_t i = threadIdx.x; i <= c.n; i += blockDim.x) {
+            const_cast<uint32_t*>(s_succ_start)[i] = (uint32_t)__ldg(&c.succ_start[i]);
+            const_cast<uint32_t*>(s_pred_start)[i] = (uint32_t)__ldg(&c.pred_start[i]);
+            if (i < c.n) const_cast<MemT*>(s_m)[i] = (MemT)__ldg(&c.m[i]);
+        }
+        for (int32_t i = threadIdx.x; i < E; i += blockDim.x) {
+            const_cast<uint16_t*>(s_succ)[i] = (uint16_t)__ldg(&c.succ[i]);
+            const_cast<uint16_t*>(s_pred)[i] = (uint16_t)__ldg(&c.pred[i]);
+        }
+        __syncthreads();
+    }
+    auto g_succ_start = [&](int32_t v) -> int32_t { return kGraphOnChip ? (int32_t)s_succ_start[v] : __ldg(&c.succ_start[v]); };
+    auto g_pred_start = [&](int32_t v) -> int32_t { return kGraphOnChip ? (int32_t)s_pred_start[v] : __ldg(&c.pred_start[v]); };
+    auto g_succ = [&](int32_t k) -> int32_t { return kGraphOnChip ? (int32_t)s_succ[k] : __ldg(&c.succ[k]); };
+    auto g_pred = [&](int32_t k) -> int32_t { return kGraphOnChip ? (int32_t)s_pred[k] : __ldg(&c.pred[k]); };
+    auto g_m = [&](int32_t v) -> MemT { return kGraphOnChip ? s_m[v] : (MemT)__ldg(&c.m[v]); };
+    char* mine = smem + (kGraphOnChip ? p.graph_bytes : 0u) + (size_t)warp * p.warp_bytes;
     uint32_t* occ = reinterpret_cast<uint32_t*>(mine);
     uint16_t* fre = reinterpret_cast<uint16_t*>(mine + p.fre_b);
     MemT* prof = reinterpret_cast<MemT*>(mine + p.prof_b);
@@ -146,17 +189,17 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                 const bool x_two_ok = c.C >= 2 && (c.cap == nullptr || __ldg(&c.cap[x]) >= 2);
                 if (cnt2 >= 1 && cnt2 <= 2 && (cnt2 == 1 || x_two_ok)) {
                     out_du = pdur + __ldg(&c.w[x]) * (cnt2 - cnt);
-                    ps0 = __ldg(&c.pred_start[x]); ps1 = __ldg(&c.pred_start[x + 1]);
-                    ss0 = __ldg(&c.succ_start[x]); ss1 = __ldg(&c.succ_start[x + 1]);
+                    ps0 = g_pred_start(x); ps1 = g_pred_start(x + 1);
+                    ss0 = g_succ_start(x); ss1 = g_succ_start(x + 1);
                     // ---- precedence (Eq. 5) can only break on edges that touch x: no first copy of a
                     // predecessor behind the first copy of x, no first copy of a successor in front of it
                     bool viol = false;
                     for (int32_t k = ps0; k < ps1; ++k) {
-                        const uint32_t wv = occ[__ldg(&c.pred[k])];
+                        const uint32_t wv = occ[g_pred(k)];
                         viol |= (int32_t)min(wv & 0xFFFFu, wv >> 16) > ta0;
                     }
                     for (int32_t k = ss0; k < ss1; ++k) {
-                        const uint32_t wv = occ[__ldg(&c.succ[k])];
+                        const uint32_t wv = occ[g_succ(k)];
                         viol |= (int32_t)min(wv & 0xFFFFu, wv >> 16) < tb0;
                     }
                     if (viol) out_st = -1;
@@ -201,7 +244,7 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                         const uint32_t seed = (uint32_t)(ta - tb) & 0xFFFFu;
                         uint32_t G = seed | seed << 16, m2 = 0;
                         for (int32_t z = s0; z < s1; ++z) {
-                            const int32_t v = __ldg(&c.succ[z]);
+                            const int32_t v = g_succ(z);
                             const uint32_t wv = v == x ? 0u : occ[v];          // the copies of x are added in child steps
                             G = __viaddmax_u16x2(wv, nbb, G);
                             m2 = max_u16x2(m2, wv);
@@ -210,7 +253,7 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                         R = ((uint32_t)tb + max(G & 0xFFFFu, G >> 16)) & 0xFFFFu;
                     };
                     {   // ---- x itself: its child copies against the copies of its successors
-                        const MemT mxv = (MemT)__ldg(&c.m[x]);
+                        const MemT mxv = g_m(x);
                         const int32_t n0 = c0, n1 = c1 == kEditNone ? c0 : c1;
                         const bool two = c1 != kEditNone;
                         uint32_t mx, R;
@@ -229,15 +272,15 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                         if (two) emit(n1, f1, mxv);
                     }
                     for (int32_t k = ps0; k < ps1; ++k) {                   // ---- the predecessors of x
-                        const int32_t y = __ldg(&c.pred[k]);
-                        const MemT my = (MemT)__ldg(&c.m[y]);
+                        const int32_t y = g_pred(k);
+                        const MemT my = g_m(y);
                         const uint32_t wy = occ[y];
                         const int32_t ya1 = (int32_t)min(wy & 0xFFFFu, wy >> 16), yb1 = (int32_t)max(wy & 0xFFFFu, wy >> 16);
                         const int32_t ya = ya1 - 1, yb = yb1 - 1;
                         const bool two = ya != yb;
                         const int32_t n0 = map(ya), n1 = map(yb);
                         uint32_t mx, R;
-                        scan_succ(__ldg(&c.succ_start[y]), __ldg(&c.succ_start[y + 1]), ya1, yb1, mx, R);
+                        scan_succ(g_succ_start(y), g_succ_start(y + 1), ya1, yb1, mx, R);
                         int32_t f1 = map(max((int32_t)mx, yb1) - 1);          // consumers other than x, in parent order
                         int32_t f0 = map((int32_t)R - 1);                     // R = ya1 when none lies between the copies
                         f1 = max(f1, c1 == kEditNone ? c0 : c1);              // x consumes y
@@ -262,11 +305,11 @@ __global__ void __launch_bounds__(kScoreThreads) search_score_kernel(const Score
                     if (ji != kEditNone) {
                         if (ji + 1 < Tc) {
                             const int32_t tr = inv(ji + 1), tl = ji >= 1 ? inv(ji - 1) : -1;
-                            cross = prof[tr] - (MemT)__ldg(&c.m[__ldg(g_row + tr)]);
-                            if (qd != kEditNone && qd > tl && qd < tr && (int32_t)fre[qd] >= tr) cross -= (MemT)__ldg(&c.m[x]);
+                            cross = prof[tr] - g_m(__ldg(g_row + tr));
+                            if (qd != kEditNone && qd > tl && qd < tr && (int32_t)fre[qd] >= tr) cross -= g_m(x);
                         } else {
                             cross = (MemT)c.sink_m;
-                            if (x_sink && qd == xb) cross -= (MemT)__ldg(&c.m[x]);
+                            if (x_sink && qd == xb) cross -= g_m(x);
                         }
                     }
                     // the parent's maxima outside the window
