@@ -241,8 +241,9 @@ int moc_check_intervals(const moc_graph* g, const int32_t* s, const int32_t* e, 
  * The cache refers to the graph handle, which must outlive it.  A call of moc_graph_set_max_copies or
  * moc_graph_set_node_caps makes the cached parents stale: moc_eval_edits (and a moc_search_run that scores
  * its proposals from a cache) then fails with MOC_ERR_ARG until moc_cache_build has run again; a changed
- * C needs a new cache.  The cache owns about 12 + 12*sizeof(sum type) bytes per step and parent of device memory, allocated by
- * moc_cache_create only.
+ * C needs a new cache.  The cache owns, per parent, 4 + 3 * (4 or 8) bytes for each of its C*n possible steps
+ * (sequence and free steps in 16 bits, usage and its prefix and suffix maxima in 32 or 64 bits as the graph's
+ * sums need) and 4 bytes per node, all allocated by moc_cache_create.
  */
 typedef struct moc_cache moc_cache; /* opaque */
 

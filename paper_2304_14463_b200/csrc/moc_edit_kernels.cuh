@@ -11,7 +11,8 @@
 // Restricted to C <= 2 (the paper's setting, Section 4.3) and sequences shorter than 65535 steps.
 //
 // Cache of one parent (all in 0-based steps; S = row stride):
-//   row[S]   the sequence                      fre[S]   free step of the copy run at each step
+//   row[S16] the sequence                      fre[S16] free step of the copy run at each step
+//            (both 16 bits per step, S16 = S rounded up to a multiple of 8 so that rows start on 16 bytes)
 //   prof[S]  memory in use at each step        pm[S]    max prof[0..t]      sm[S]  max prof[t..T-1]
 //   occ[n]   the two steps of every node, 1-based, 16 bits each (equal when the node runs once)
 //   len, status, peak, dur
@@ -27,6 +28,7 @@ constexpr int kEditThreads = 256;   // 8 warps per block, one parent or one edit
 
 struct EditCacheDev {
     int32_t n, C, P, stride, occ_stride;
+    int32_t stride16;           // row stride of the 16-bit arrays row and fre
     int32_t max_T;              // C * n
     const int32_t* succ_start;  // successor and predecessor lists (CSR)
     const int32_t* succ;
@@ -36,8 +38,8 @@ struct EditCacheDev {
     const int64_t* m;
     const int32_t* cap;         // per-node caps or nullptr
     int64_t sink_m;             // sum of m over the nodes without successors
-    int32_t* row;
-    int32_t* fre;
+    uint16_t* row;
+    uint16_t* fre;
     void* prof;                 // MemT [P][stride]
     void* pm;
     void* sm;
@@ -141,7 +143,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
         const int32_t T = p.lens[b];
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;
-        int32_t* row = c.row + (int64_t)b * c.stride;
+        uint16_t* row = c.row + (int64_t)b * c.stride16;
         if (T >= n && T <= c.max_T) {
             for (int32_t i = lane; i < wstride; i += 32) word[i] = 0;
             for (int32_t i = lane; i < c.stride + 4; i += 32) arrA[i] = 0;
@@ -149,7 +151,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
             // ---- occurrence words (1-based steps, 16 bits each) and the copy of the row
             const int32_t* src = p.seqs + p.offs[b];
             auto put = [&](int32_t v, int32_t t) {
-                row[t] = v;
+                row[t] = (uint16_t)v;
                 const uint32_t slot = min((uint32_t)v, (uint32_t)n);      // ids outside [0, n) land in a spare word
                 const uint32_t t1 = (uint32_t)t + 1u;
                 const uint32_t old = atomicExch(&word[slot], t1 * 0x10001u);
@@ -168,7 +170,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
             uint32_t vsum = 0;
             bool absent = false, dep = false, over = false;
             int64_t dur = 0;
-            int32_t* fre = c.fre + (int64_t)b * c.stride;
+            uint16_t* fre = c.fre + (int64_t)b * c.stride16;
             if (p.n_tiles > 0) {
                 // The node pass of the evaluation kernel: lane l serves the nodes l (mod 32) in tiles of two
                 // slots, successor rows of packed word offsets, two shifted packed reductions per successor
@@ -255,7 +257,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                 over = __any_sync(kFull, (int32_t)capw < 0) || (int)((acc_all >> kPairCntShift) & 0x7FFFu) != T - n;
                 dep = (depw & 0x80008000u) != 0;
                 __syncwarp();
-                for (int32_t t = lane; t < T; t += 32) fre[t] = (int32_t)arrB[t];
+                for (int32_t t = lane; t < T; t += 32) fre[t] = (uint16_t)arrB[t];
                 // position sum and duration in the form the rest of the kernel expects
                 vsum = lane == 0 ? (uint32_t)T * ((uint32_t)T + 1u) / 2u : 0u;
                 dur = lane == 0 ? p.base_dur + (int64_t)(acc_all & kPairDurMask) : 0;
@@ -282,11 +284,11 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                 }
                 if (a != 0) {
                     const MemT mu = (MemT)__ldg(&c.m[u]);
-                    fre[bp - 1] = (int32_t)fb - 1;
+                    fre[bp - 1] = (uint16_t)(fb - 1);
                     edit_add(&arrA[bp - 1], mu);
                     edit_add(&arrA[fb], (MemT)(-mu));
                     if (a != bp) {
-                        fre[a - 1] = (int32_t)fa - 1;
+                        fre[a - 1] = (uint16_t)(fa - 1);
                         edit_add(&arrA[a - 1], mu);
                         edit_add(&arrA[fa], (MemT)(-mu));
                     }
@@ -404,13 +406,13 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
         }
         if (go) go = o >= 0 && o <= 2 && qq >= 0 && qq < T && (o == 1 || (jj >= 0 && jj <= (o == 0 ? T : T - 1)));
         if (go) {
-            const int32_t* row = c.row + (int64_t)ci * c.stride;
-            const int32_t* fre = c.fre + (int64_t)ci * c.stride;
+            const uint16_t* row = c.row + (int64_t)ci * c.stride16;
+            const uint16_t* fre = c.fre + (int64_t)ci * c.stride16;
             const MemT* prof = reinterpret_cast<const MemT*>(c.prof) + (int64_t)ci * c.stride;
             const MemT* pmx = reinterpret_cast<const MemT*>(c.pm) + (int64_t)ci * c.stride;
             const MemT* smx = reinterpret_cast<const MemT*>(c.sm) + (int64_t)ci * c.stride;
             const uint32_t* occ = c.occ + (int64_t)ci * c.occ_stride;
-            const int32_t x = row[qq];
+            const int32_t x = (int32_t)row[qq];
             const int32_t qd = o >= 1 ? qq : kEditNone, ji = o != 1 ? jj : kEditNone;
             const int32_t Tc = T + (o == 0 ? 1 : 0) - (o == 1 ? 1 : 0);
             auto map = [&](int32_t s) -> int32_t { const int32_t s1 = s - (s > qd ? 1 : 0); return s1 + (s1 >= ji ? 1 : 0); };
@@ -504,20 +506,20 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
                         };
                         if (y == x) {
                             int32_t l, h;
-                            old_range(xa, fre[xa], x_sink && cnt == 1, l, h);
+                            old_range(xa, (int32_t)fre[xa], x_sink && cnt == 1, l, h);
                             emit(l, h, (MemT)(-my));
                             if (cnt == 2) {
-                                old_range(xb, fre[xb], x_sink, l, h);
+                                old_range(xb, (int32_t)fre[xb], x_sink, l, h);
                                 emit(l, h, (MemT)(-my));
                             }
                             emit(n0, f0, my);
                             if (two) emit(n1, f1, my);
                         } else {
                             int32_t l, h;
-                            old_range(ya, fre[ya], false, l, h);
+                            old_range(ya, (int32_t)fre[ya], false, l, h);
                             if (h != f0) emit(min(h, f0) + 1, max(h, f0), f0 > h ? my : (MemT)(-my));
                             if (yb != ya) {
-                                old_range(yb, fre[yb], false, l, h);
+                                old_range(yb, (int32_t)fre[yb], false, l, h);
                                 if (h != f1) emit(min(h, f1) + 1, max(h, f1), f1 > h ? my : (MemT)(-my));
                             }
                         }
@@ -539,8 +541,8 @@ __global__ void __launch_bounds__(kEditThreads) edit_eval_kernel(const EditParam
                     if (ji != kEditNone) {
                         if (ji + 1 < Tc) {
                             const int32_t tr = inv(ji + 1), tl = ji >= 1 ? inv(ji - 1) : -1;
-                            cross = prof[tr] - (MemT)__ldg(&c.m[row[tr]]);
-                            if (qd != kEditNone && qd > tl && qd < tr && fre[qd] >= tr) cross -= (MemT)__ldg(&c.m[x]);
+                            cross = prof[tr] - (MemT)__ldg(&c.m[(int32_t)row[tr]]);
+                            if (qd != kEditNone && qd > tl && qd < tr && (int32_t)fre[qd] >= tr) cross -= (MemT)__ldg(&c.m[x]);
                         } else {
                             cross = (MemT)c.sink_m;
                             if (x_sink && qd == xb) cross -= (MemT)__ldg(&c.m[x]);

@@ -68,7 +68,7 @@ int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
     h->max_parents = max_parents;
     h->wide = g->sum_m > (int64_t)INT32_MAX / g->C;
     const size_t msz = h->wide ? 8 : 4;
-    const int32_t stride = (int32_t)((max_T + 3) & ~int64_t(3)), occ_stride = (g->n + 1 + 3) & ~3;
+    const int32_t stride = (int32_t)((max_T + 3) & ~int64_t(3)), occ_stride = (g->n + 1 + 3) & ~3, stride16 = (stride + 7) & ~7;
     h->warp_bytes = moc::edit_warp_bytes(g->n, stride, msz);
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
     if (h->warp_bytes > cap) {
@@ -83,8 +83,8 @@ int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
         if (fit > best) { best = fit; h->wpb = k; }
     }
     h->grid_cap = g->sm_count * std::max(1, best / h->wpb);
-    const size_t P = (size_t)max_parents, S = (size_t)stride;
-    const size_t o_row = 0, o_fre = o_row + up256(P * S * 4), o_prof = o_fre + up256(P * S * 4), o_pm = o_prof + up256(P * S * msz),
+    const size_t P = (size_t)max_parents, S = (size_t)stride, S16 = (size_t)stride16;
+    const size_t o_row = 0, o_fre = o_row + up256(P * S16 * 2), o_prof = o_fre + up256(P * S16 * 2), o_pm = o_prof + up256(P * S * msz),
                  o_sm = o_pm + up256(P * S * msz), o_occ = o_sm + up256(P * S * msz), o_len = o_occ + up256(P * occ_stride * 4),
                  o_st = o_len + up256(P * 4), o_peak = o_st + up256(P * 4), o_dur = o_peak + up256(P * 8),
                  o_offs = o_dur + up256(P * 8), total = o_offs + up256((P + 1) * 8);
@@ -101,6 +101,7 @@ int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
     c.P = 0;
     c.stride = stride;
     c.occ_stride = occ_stride;
+    c.stride16 = stride16;
     c.max_T = (int32_t)max_T;
     c.succ_start = g->d_succ_start;
     c.succ = g->d_succ;
@@ -110,8 +111,8 @@ int moc_cache_create(const moc_graph* g, int32_t max_parents, moc_cache** out) {
     c.m = g->d_m64;
     c.cap = g->d_cap;
     c.sink_m = g->sink_m;
-    c.row = (int32_t*)(b + o_row);
-    c.fre = (int32_t*)(b + o_fre);
+    c.row = (uint16_t*)(b + o_row);
+    c.fre = (uint16_t*)(b + o_fre);
     c.prof = b + o_prof;
     c.pm = b + o_pm;
     c.sm = b + o_sm;

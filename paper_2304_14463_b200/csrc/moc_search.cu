@@ -50,8 +50,8 @@ bool plan_fused(moc_search* s) {
     moc::ScoreParams& sp = s->sp;
     const size_t msz = h->wide ? 8 : 4;
     const int32_t worst = 4 + 2 * g->max_indeg;
-    sp.list_cap = std::max(192, (worst + 31) & ~31);
-    sp.warp_bytes = (uint32_t)moc::score_warp_bytes(h->c.occ_stride, h->c.stride, msz, sp.list_cap, &sp.fre_b, &sp.prof_b,
+    sp.list_cap = std::max(128, (worst + 31) & ~31);
+    sp.warp_bytes = (uint32_t)moc::score_warp_bytes(h->c.occ_stride, h->c.stride, msz, sp.list_cap, &sp.fre_b, &sp.row_b, &sp.prof_b,
                                                    &sp.lh_b, &sp.val_b, &sp.diff_b);
     const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
     if ((size_t)sp.warp_bytes * 4 > cap) return false;

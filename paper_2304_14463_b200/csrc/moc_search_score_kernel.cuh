@@ -36,17 +36,19 @@ struct ScoreParams {
     uint32_t graph_bytes;   // shared memory of the block's copy of the graph (kGraphOnChip), a multiple of 16
     uint32_t gs_pred_b, gs_m_b, gs_succ_b, gs_predl_b;   // its parts after the successor offsets
     uint32_t warp_bytes;    // shared memory of one warp
-    uint32_t fre_b, prof_b, lh_b, val_b, diff_b;   // byte offsets of its parts (copy positions come first)
+    uint32_t fre_b, row_b, prof_b, lh_b, val_b, diff_b;   // byte offsets of its parts (copy positions come first)
     int32_t list_cap;
 };
 
-// Bytes of one warp: copy positions (occ_stride words), free steps (16 bits each), profile, range list,
-// difference array of the corrections (stride + 4 entries).
+// Bytes of one warp: copy positions (occ_stride words), free steps and the sequence (16 bits each), profile,
+// range list, difference array of the corrections (stride + 4 entries).
 __host__ __device__ inline size_t score_warp_bytes(int32_t occ_stride, int32_t stride, size_t mem_sz, int32_t list_cap,
-                                                   uint32_t* fre_b, uint32_t* prof_b, uint32_t* lh_b, uint32_t* val_b,
-                                                   uint32_t* diff_b) {
+                                                   uint32_t* fre_b, uint32_t* row_b, uint32_t* prof_b, uint32_t* lh_b,
+                                                   uint32_t* val_b, uint32_t* diff_b) {
     size_t o = (size_t)occ_stride * 4;
     *fre_b = (uint32_t)o;
+    o += ((size_t)stride * 2 + 15) & ~size_t(15);          // = 2 * stride16
+    *row_b = (uint32_t)o;
     o += ((size_t)stride * 2 + 15) & ~size_t(15);
     *prof_b = (uint32_t)o;
     o += ((size_t)stride * mem_sz + 15) & ~size_t(15);
@@ -73,6 +75,11 @@ __host__ __device__ inline size_t score_graph_bytes(int32_t n, int64_t n_edges, 
     *predl_b = (uint32_t)o;
     o += ((size_t)n_edges * 2 + 15) & ~size_t(15);
     return o;
+}
+
+// 16 bytes from global to shared memory without a register in between (completed by cp.async.wait_all).
+__device__ __forceinline__ void score_copy16(void* dst_shared, const void* src_global) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)), "l"(src_global) : "memory");
 }
 
 // kGraphOnChip: the block keeps the graph's lists and output sizes in shared memory (every lane walks them
@@ -110,6 +117,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
     char* mine = smem + (kGraphOnChip ? p.graph_bytes : 0u) + (size_t)warp * p.warp_bytes;
     uint32_t* occ = reinterpret_cast<uint32_t*>(mine);
     uint16_t* fre = reinterpret_cast<uint16_t*>(mine + p.fre_b);
+    uint16_t* row = reinterpret_cast<uint16_t*>(mine + p.row_b);
     MemT* prof = reinterpret_cast<MemT*>(mine + p.prof_b);
     MemT* rv = reinterpret_cast<MemT*>(mine + p.val_b);
     uint32_t* rl = reinterpret_cast<uint32_t*>(mine + p.lh_b);
@@ -123,21 +131,23 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
     for (int32_t ci = blockIdx.x * wpb + warp; ci < s.P; ci += gridDim.x * wpb) {
         const int32_t T = c.len[ci], pst = c.status[ci];
         const int64_t pdur = c.dur[ci];
-        const int32_t* g_row = c.row + (int64_t)ci * c.stride;
         const MemT* g_pm = reinterpret_cast<const MemT*>(c.pm) + (int64_t)ci * c.stride;
         const MemT* g_sm = reinterpret_cast<const MemT*>(c.sm) + (int64_t)ci * c.stride;
-        // ---- stage the chain's cache entry: copy positions, free steps (16 bits), profile
+        // ---- stage the chain's cache entry (copy positions, profile, free steps, sequence): asynchronous
+        // 16-byte copies, all in flight at once
         {
             const uint4* g_occ = reinterpret_cast<const uint4*>(c.occ + (int64_t)ci * c.occ_stride);
-            for (int32_t i = lane; i < c.occ_stride / 4; i += 32) reinterpret_cast<uint4*>(occ)[i] = g_occ[i];
-            const int4* g_fre = reinterpret_cast<const int4*>(c.fre + (int64_t)ci * c.stride);
-            for (int32_t i = lane; i < (T + 3) / 4; i += 32) {
-                const int4 v = g_fre[i];
-                reinterpret_cast<uint2*>(fre)[i] = make_uint2((uint32_t)v.x | (uint32_t)v.y << 16, (uint32_t)v.z | (uint32_t)v.w << 16);
-            }
+            for (int32_t i = lane; i < c.occ_stride / 4; i += 32) score_copy16(reinterpret_cast<uint4*>(occ) + i, g_occ + i);
             const uint4* g_prof = reinterpret_cast<const uint4*>(reinterpret_cast<const MemT*>(c.prof) + (int64_t)ci * c.stride);
             constexpr int32_t kPer = 16 / (int32_t)sizeof(MemT);
-            for (int32_t i = lane; i < (T + kPer - 1) / kPer; i += 32) reinterpret_cast<uint4*>(prof)[i] = g_prof[i];
+            for (int32_t i = lane; i < (T + kPer - 1) / kPer; i += 32) score_copy16(reinterpret_cast<uint4*>(prof) + i, g_prof + i);
+            const uint4* g_fre = reinterpret_cast<const uint4*>(c.fre + (int64_t)ci * c.stride16);
+            const uint4* g_row = reinterpret_cast<const uint4*>(c.row + (int64_t)ci * c.stride16);
+            for (int32_t i = lane; i < (T + 7) / 8; i += 32) {
+                score_copy16(reinterpret_cast<uint4*>(fre) + i, g_fre + i);
+                score_copy16(reinterpret_cast<uint4*>(row) + i, g_row + i);
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
         }
         __syncwarp();
 
@@ -159,7 +169,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
             bool go = live && qq < T;
             if (go && pst < 0) { out_st = kStatusParentInvalid; go = false; }
             // ---- per proposal: the edit in parent and child steps
-            const int32_t x = go ? __ldg(g_row + qq) : 0;
+            const int32_t x = go ? (int32_t)row[qq] : 0;
             const int32_t qd = o >= 1 ? qq : kEditNone, ji = o != 1 ? jj : kEditNone;
             const int32_t Tc = T + (o == 0 ? 1 : 0) - (o == 1 ? 1 : 0);
             auto map = [&](int32_t st) -> int32_t { const int32_t s1 = st - (st > qd ? 1 : 0); return s1 + (s1 >= ji ? 1 : 0); };
@@ -305,7 +315,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                     if (ji != kEditNone) {
                         if (ji + 1 < Tc) {
                             const int32_t tr = inv(ji + 1), tl = ji >= 1 ? inv(ji - 1) : -1;
-                            cross = prof[tr] - g_m(__ldg(g_row + tr));
+                            cross = prof[tr] - g_m((int32_t)row[tr]);
                             if (qd != kEditNone && qd > tl && qd < tr && (int32_t)fre[qd] >= tr) cross -= g_m(x);
                         } else {
                             cross = (MemT)c.sink_m;
@@ -385,9 +395,22 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                 const int32_t cur = s.cur[ci];
                 const int32_t qd = op >= 1 ? q : INT32_MAX, ji = op != 1 ? j : INT32_MAX;
                 const int32_t Tc = T + (op == 0 ? 1 : 0) - (op == 1 ? 1 : 0);
-                const int64_t src_off = ((int64_t)cur * s.P + ci) * s.stride, dst_off = ((int64_t)(cur ^ 1) * s.P + ci) * s.stride;
-                const int32_t x = __ldg(s.rows + src_off + q);
-                search_write_edited(s.rows + src_off, s.rows + dst_off, Tc, qd, ji, x, lane);
+                const int64_t dst_off = ((int64_t)(cur ^ 1) * s.P + ci) * s.stride;
+                // the edited copy of the staged sequence: element qd out, x in front of index ji of what is left
+                const int32_t x = (int32_t)row[q];
+                int32_t* dst = s.rows + dst_off;
+                auto at = [&](int32_t i) -> int32_t {
+                    if (i == ji) return x;
+                    const int32_t k = i - (i > ji ? 1 : 0);
+                    return (int32_t)row[k + (k >= qd ? 1 : 0)];
+                };
+                for (int32_t i0 = 4 * lane; i0 < Tc; i0 += 128) {
+                    if (i0 + 4 <= Tc) {
+                        *reinterpret_cast<int4*>(dst + i0) = make_int4(at(i0), at(i0 + 1), at(i0 + 2), at(i0 + 3));
+                    } else {
+                        for (int32_t i = i0; i < Tc; ++i) dst[i] = at(i);
+                    }
+                }
                 __syncwarp();
                 if (lane == 0) {
                     s.cur[ci] = cur ^ 1;

@@ -262,8 +262,8 @@ def _layered_dense(width, layers, seed):
 
 
 def test_search_chain_kernel_in_rounds(B):
-    """In-degree 30: one proposal may need 64 entries of the 192-entry correction list of a warp, so a pass with
-    more than three admissible proposals is scored in several rounds.  A copy inserted behind the node's first one
+    """In-degree 30: one proposal may need 64 entries of the 128-entry correction list of a warp, so a pass with
+    more than two admissible proposals is scored in several rounds.  A copy inserted behind the node's first one
     is always admissible, so with inserts only about half of the 32 proposals of a pass are."""
     n, edges, w, m = _layered_dense(30, 3, 2)
     rng = np.random.default_rng(3)
