@@ -452,7 +452,7 @@ def run_edits(args):
             "dtype": "int64" if msz == 8 else "int32", "data": "synthetic",
             "config": {"workload": f"moc_eval_edits on {base.name}: n={base.n} C={base.C}, {P} cached parents, {per_parent} random "
                                    f"edits each (insert / delete / move), M={PCT}% of no-remat peak",
-                       "cold_l2": f"cache of the parents: {P * (12 + 3 * msz) * (2 * base.n) / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
+                       "cold_l2": f"cache of the parents: {P * (4 + 3 * msz) * (2 * base.n) / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
                        "mean_T": mean_T, "mean_recomputed_steps": mean_window},
             "equivalent_schedule_steps_per_s": nE * mean_T / (ms * 1e-3), "cache_build_ms": build_ms, "gpu_launches": steps,
             "admissible_only": None if adm_ms is None else {
@@ -462,8 +462,8 @@ def run_edits(args):
             "status_counts": {str(k): int((st == k).sum()) for k in (1, 0, -1, -2, -3)},
             "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
                          "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak_gbs, "peak_kind": f"of {peak_kind}",
-                         "traffic": 116593664 + 8356352,
-                         "traffic_source": "ncu, one launch of this workload: dram read 116.59 MB, write 8.36 MB",
+                         "traffic": 104447232 + 4538112,
+                         "traffic_source": "ncu, one launch of this workload: dram read 104.45 MB, write 4.54 MB",
                          "algorithmic_bytes_per_launch": alg_bytes},
             "clocks": clocks.summary()}
     if not args.no_cpu_baseline:
