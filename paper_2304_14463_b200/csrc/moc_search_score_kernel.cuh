@@ -82,6 +82,9 @@ __device__ __forceinline__ void score_copy16(void* dst_shared, const void* src_g
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)), "l"(src_global) : "memory");
 }
 
+__device__ __forceinline__ int32_t score_warp_max(int32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
+__device__ __forceinline__ int64_t score_warp_max(int64_t v) { return edit_warp_max(v); }
+
 // kGraphOnChip: the block keeps the graph's lists and output sizes in shared memory (every lane walks them
 // at its own node, and what the warps' arrays leave of the L1 is too small to hold them).
 template <typename MemT, bool kGraphOnChip>
@@ -346,10 +349,10 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                     const int32_t L = hi - lo + 1;
                     const int32_t per = ((L + 31) / 32) | 1;
                     const int32_t t0 = lo + min(L, lane * per), t1 = lo + min(L, (lane + 1) * per);
-                    MemT sum = 0;
-                    for (int32_t t = t0; t < t1; ++t) sum += diff[t];
-                    MemT run = edit_warp_incl_sum(sum, lane) - sum;
-                    MemT top = 0;
+                    // one pass: running correction and usage relative to the start of the run, then the carry
+                    // from the runs in front (max over the run of carry + x = carry + max x)
+                    MemT run = 0, top = sizeof(MemT) == 8 ? (MemT)INT64_MIN : (MemT)INT32_MIN;
+                    const bool any = t0 < t1;
                     for (int32_t t = t0; t < t1; ++t) {
                         run += diff[t];
                         diff[t] = 0;
@@ -357,8 +360,10 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                         const MemT u = run + (t == ji_s ? cr_s : prof[tt + (tt >= qd_s ? 1 : 0)]);
                         top = u > top ? u : top;
                     }
+                    const MemT carry = edit_warp_incl_sum(run, lane) - run;
+                    top = any ? top + carry : (MemT)0;          // usage is never negative: 0 is neutral
                     if (lane == 0) diff[hi + 1] = 0;
-                    top = edit_warp_max(top);
+                    top = score_warp_max(top);
                     if (lane == sl) best = top > best ? top : best;
                     __syncwarp();
                 }
