@@ -207,10 +207,12 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                     // ---- precedence (Eq. 5) can only break on edges that touch x: no first copy of a
                     // predecessor behind the first copy of x, no first copy of a successor in front of it
                     bool viol = false;
+#pragma unroll 1
                     for (int32_t k = ps0; k < ps1; ++k) {
                         const uint32_t wv = occ[g_pred(k)];
                         viol |= (int32_t)min(wv & 0xFFFFu, wv >> 16) > ta0;
                     }
+#pragma unroll 1
                     for (int32_t k = ss0; k < ss1; ++k) {
                         const uint32_t wv = occ[g_succ(k)];
                         viol |= (int32_t)min(wv & 0xFFFFu, wv >> 16) < tb0;
@@ -256,6 +258,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                         const uint32_t ntb = (uint32_t)(-tb) & 0xFFFFu, nbb = ntb | ntb << 16;
                         const uint32_t seed = (uint32_t)(ta - tb) & 0xFFFFu;
                         uint32_t G = seed | seed << 16, m2 = 0;
+#pragma unroll 1
                         for (int32_t z = s0; z < s1; ++z) {
                             const int32_t v = g_succ(z);
                             const uint32_t wv = v == x ? 0u : occ[v];          // the copies of x are added in child steps
@@ -284,6 +287,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
                         emit(n0, f0, mxv);
                         if (two) emit(n1, f1, mxv);
                     }
+#pragma unroll 1
                     for (int32_t k = ps0; k < ps1; ++k) {                   // ---- the predecessors of x
                         const int32_t y = g_pred(k);
                         const MemT my = g_m(y);
@@ -384,13 +388,17 @@ __global__ void __launch_bounds__(kScoreThreads, 1) search_score_kernel(const Sc
         }
 
         // ---- the chain's best proposal, and whether it replaces the sequence
-        int64_t a = b_a, d = b_d;
-        int32_t be = b_e;
-        for (int off = 16; off > 0; off >>= 1) {
-            const int64_t a2 = __shfl_xor_sync(kFull, a, off), d2 = __shfl_xor_sync(kFull, d, off);
-            const int32_t e2 = __shfl_xor_sync(kFull, be, off);
-            if (a2 < a || (a2 == a && (d2 < d || (d2 == d && e2 < be)))) { a = a2; d = d2; be = e2; }
-        }
+        // smallest key (a, d) among the lanes that hold a proposal, lowest sample among equals; a, d >= 0
+        auto min64 = [&](int64_t v, bool in) -> int64_t {
+            const uint32_t hi = in ? (uint32_t)((uint64_t)v >> 32) : 0xFFFFFFFFu, hmin = __reduce_min_sync(kFull, hi);
+            const uint32_t lo = (in && hi == hmin) ? (uint32_t)v : 0xFFFFFFFFu, lmin = __reduce_min_sync(kFull, lo);
+            return (int64_t)((uint64_t)hmin << 32 | lmin);
+        };
+        const bool has = b_e != INT32_MAX;
+        const int64_t a_min = min64(b_a, has);
+        const bool has_a = has && b_a == a_min;
+        const int64_t d_min = min64(b_d, has_a);
+        const int32_t be = (int32_t)__reduce_min_sync(kFull, (has_a && b_d == d_min) ? (uint32_t)b_e : (uint32_t)INT32_MAX);
         if (be != INT32_MAX) {
             const int src = be & 31;
             const int64_t pk = __shfl_sync(kFull, b_pk, src), du = __shfl_sync(kFull, b_d, src);
