@@ -316,9 +316,9 @@ int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) 
     ip.todo = (int32_t*)(b + o_todo);
     ip.todo_count = (int32_t*)(b + o_cnt);
     MOC_CUDA(cudaMemset(ip.todo_count, 0, 8));
-    // scoring kernel: a warp per chain when asked for, or by default from four proposals per chain on
+    // scoring kernel: a warp per chain when asked for, or by default from two proposals per chain on
     s->fused = false;
-    if (incremental == MOC_SEARCH_SCORE_CHAIN || (incremental == MOC_SEARCH_SCORE_AUTO && samples >= 4)) {
+    if (incremental == MOC_SEARCH_SCORE_CHAIN || (incremental == MOC_SEARCH_SCORE_AUTO && samples >= 2)) {
         s->fused = plan_fused(s);
         if (!s->fused && incremental == MOC_SEARCH_SCORE_CHAIN) {
             cudaFree(s->d_inc);
