@@ -24,7 +24,8 @@
 
 namespace moc {
 
-constexpr int kEditThreads = 256;   // 8 warps per block, one parent or one edit per warp at a time
+constexpr int kEditThreads = 256;   // 8 warps per block, one edit per warp at a time
+constexpr int kPrepThreads = 768;   // cache build: up to 24 warps per block, one parent per warp at a time
 
 struct EditCacheDev {
     int32_t n, C, P, stride, occ_stride;
@@ -69,6 +70,10 @@ struct PrepParams {
     const uint64_t* wslot;
     const uint32_t* sell;
     int64_t base_dur;           // sum of all w
+    // chip_bytes > 0: the block first copies the tiles into its shared memory (records, then durations at
+    // chip_w_b, then successor entries at chip_sell_b; sell_len entries) and the warps' arrays follow
+    uint32_t chip_bytes, chip_w_b, chip_sell_b;
+    int32_t sell_len;
 };
 
 template <typename T>
@@ -123,13 +128,25 @@ __host__ __device__ inline size_t edit_warp_bytes(int32_t n, int32_t stride, siz
 
 // Full evaluation of every parent (same quantities as the evaluation kernels: Section 2, Eqs. 1-8)
 // that also writes the cache.  One warp per parent.
-template <typename MemT>
-__global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepParams p) {
+template <typename MemT, bool kChip>
+__global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepParams p) {
     extern __shared__ __align__(16) char smem[];
     const EditCacheDev& c = p.c;
     const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
-    char* ws = smem + (size_t)warp * p.warp_bytes;
+    if (kChip) {
+        // what the L1 keeps of the tiles between parents is little beside the warps' arrays: the block holds its own copy
+        const uint32_t rec_v = (sizeof(MemT) == 4 ? 8u : 16u) * 64u * (uint32_t)p.n_tiles / 16u, w_v = 8u * 64u * (uint32_t)p.n_tiles / 16u;
+        const uint32_t sell_v = ((uint32_t)p.sell_len * 4u + 15u) / 16u;
+        const uint4* g_rec = reinterpret_cast<const uint4*>(p.rec);
+        const uint4* g_w = reinterpret_cast<const uint4*>(p.wslot);
+        const uint4* g_sell = reinterpret_cast<const uint4*>(p.sell);
+        for (uint32_t i = threadIdx.x; i < rec_v; i += blockDim.x) reinterpret_cast<uint4*>(smem)[i] = __ldg(g_rec + i);
+        for (uint32_t i = threadIdx.x; i < w_v; i += blockDim.x) reinterpret_cast<uint4*>(smem + p.chip_w_b)[i] = __ldg(g_w + i);
+        for (uint32_t i = threadIdx.x; i < sell_v; i += blockDim.x) reinterpret_cast<uint4*>(smem + p.chip_sell_b)[i] = __ldg(g_sell + i);
+        __syncthreads();
+    }
+    char* ws = smem + (kChip ? p.chip_bytes : 0u) + (size_t)warp * p.warp_bytes;
     uint32_t* word = reinterpret_cast<uint32_t*>(ws);
     const size_t arr_bytes = (((size_t)c.stride + 4) * sizeof(MemT) + 15) & ~size_t(15);
     const int32_t n = c.n, wstride = edit_word_stride(c.n);
@@ -177,9 +194,11 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                 // word (end of the last copy with the precedence test, end of the first copy).
                 constexpr uint32_t kRecB = sizeof(MemT) == 4 ? 8u : 16u;
                 const uint32_t wa = (uint32_t)__cvta_generic_to_shared(word);
-                const char* prec = reinterpret_cast<const char*>(p.rec) + kRecB * lane;
-                const uint64_t* pw = p.wslot + lane;
-                const uint32_t* ps = p.sell + lane;
+                const char* prec = (kChip ? smem : reinterpret_cast<const char*>(p.rec)) + kRecB * lane;
+                const uint64_t* pw = (kChip ? reinterpret_cast<const uint64_t*>(smem + p.chip_w_b) : p.wslot) + lane;
+                const uint32_t* ps = (kChip ? reinterpret_cast<const uint32_t*>(smem + p.chip_sell_b) : p.sell) + lane;
+                auto ld32 = [&](const uint32_t* q) -> uint32_t { return kChip ? lds_u32_nv((uint32_t)__cvta_generic_to_shared(q)) : __ldg(q); };
+                auto ld64 = [&](const uint64_t* q) -> uint64_t { return kChip ? lds_u64((uint32_t)__cvta_generic_to_shared(q)) : __ldg(q); };
                 uint32_t vmin = 0xFFFFFFFFu, depw = 0, capw = 0;
                 uint64_t acc = 0;
                 const uint32_t empty_off = 4u * (((uint32_t)n + 2u + 3u) & ~3u);   // where the records of empty slots point
@@ -196,11 +215,13 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                     for (int h = 0; h < 2; ++h) {
                         uint32_t x;
                         if constexpr (sizeof(MemT) == 4) {
-                            const uint2 r = __ldg(reinterpret_cast<const uint2*>(prec + 32 * kRecB * h));
+                            const uint2 r = kChip ? lds_v2((uint32_t)__cvta_generic_to_shared(prec + 32 * kRecB * h))
+                                                  : __ldg(reinterpret_cast<const uint2*>(prec + 32 * kRecB * h));
                             x = r.x;
                             mm[h] = (MemT)r.y;
                         } else {
-                            const uint4 r = __ldg(reinterpret_cast<const uint4*>(prec + 32 * kRecB * h));
+                            const uint4 r = kChip ? lds_v4((uint32_t)__cvta_generic_to_shared(prec + 32 * kRecB * h))
+                                                  : __ldg(reinterpret_cast<const uint4*>(prec + 32 * kRecB * h));
                             x = r.x;
                             mm[h] = (MemT)((uint64_t)r.z | ((uint64_t)r.w << 32));
                         }
@@ -217,10 +238,10 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                         Gb[h] = 0x00010000u - Ga[h];
                     }
                     rows = __shfl_sync(kFull, rows, 0);
-                    uint32_t e_next = rows > 0 ? __ldg(ps) : 0u;           // one row ahead: the tiles come through L1
+                    uint32_t e_next = rows > 0 ? ld32(ps) : 0u;            // one row ahead
                     for (int k = 0; k < rows; ++k, ps += 32) {
                         const uint32_t e = e_next;
-                        if (k + 1 < rows) e_next = __ldg(ps + 32);
+                        if (k + 1 < rows) e_next = ld32(ps + 32);
                         const uint32_t r0 = lds_u32(wa + (e & 0xFFFFu)), r1 = lds_u32(wa + (e >> 16));
                         Ga[0] = __viaddmax_u16x2(r0, naa[0], Ga[0]);
                         Ga[1] = __viaddmax_u16x2(r1, naa[1], Ga[1]);
@@ -242,7 +263,7 @@ __global__ void __launch_bounds__(kEditThreads) edit_prepare_kernel(const PrepPa
                                 arrB[a16 - 1] = (MemT)fa - 1;
                                 edit_add(&arrA[a16 - 1], mm[h]);
                                 edit_add(&arrA[fa], (MemT)(-mm[h]));
-                                const uint64_t wx = __ldg(pw + 32 * h);
+                                const uint64_t wx = ld64(pw + 32 * h);
                                 capw |= (uint32_t)(wx >> 32);
                                 acc += wx;
                             }

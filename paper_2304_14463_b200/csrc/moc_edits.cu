@@ -41,10 +41,27 @@ int cache_prepare(moc_cache* h, const int32_t* seqs, const int32_t* lens, const 
     p.wslot = g->d_wslot;
     p.sell = g->d_sell;
     p.base_dur = g->sum_w;
-    auto fn = h->wide ? moc::edit_prepare_kernel<int64_t> : moc::edit_prepare_kernel<int32_t>;
-    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(h->g->smem_optin - 1024)));
-    const int grid = (int)std::min<int64_t>(h->grid_cap, ((int64_t)P + h->wpb - 1) / h->wpb);
-    fn<<<grid, 32 * h->wpb, h->warp_bytes * h->wpb, st>>>(p);
+    // block shape: with the tiles in the block's shared memory when that keeps at least 12 warps on an SM
+    const size_t optin = g->smem_optin, cap = optin > 2048 ? optin - 2048 : 0;
+    const size_t rec_b = (h->wide ? 16 : 8) * 64 * (size_t)g->n_tiles, w_b = 8 * 64 * (size_t)g->n_tiles,
+                 sell_b = (4 * (size_t)g->sell_len + 15) & ~size_t(15), chip_b = rec_b + w_b + sell_b;
+    int wpb = h->wpb, grid_cap = h->grid_cap;
+    bool chip = false;
+    if (tiles && chip_b + 12 * h->warp_bytes <= cap) {
+        chip = true;
+        wpb = (int)std::min<size_t>(moc::kPrepThreads / 32, (cap - chip_b) / h->warp_bytes);
+        grid_cap = g->sm_count;
+        p.chip_bytes = (uint32_t)chip_b;
+        p.chip_w_b = (uint32_t)rec_b;
+        p.chip_sell_b = (uint32_t)(rec_b + w_b);
+        p.sell_len = g->sell_len;
+    }
+    const void* fn = chip ? (h->wide ? (const void*)moc::edit_prepare_kernel<int64_t, true> : (const void*)moc::edit_prepare_kernel<int32_t, true>)
+                          : (h->wide ? (const void*)moc::edit_prepare_kernel<int64_t, false> : (const void*)moc::edit_prepare_kernel<int32_t, false>);
+    MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(optin - 1024)));
+    const int grid = (int)std::min<int64_t>(grid_cap, ((int64_t)P + wpb - 1) / wpb);
+    void* args[] = {&p};
+    MOC_CUDA(cudaLaunchKernel(fn, dim3(grid), dim3(32 * wpb), args, (chip ? chip_b : 0) + h->warp_bytes * wpb, st));
     MOC_CUDA(cudaGetLastError());
     return MOC_OK;
 }
