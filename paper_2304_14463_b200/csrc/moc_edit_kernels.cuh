@@ -155,9 +155,18 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
     constexpr uint32_t kFull = 0xFFFFFFFFu;
 
     const int32_t count = p.todo != nullptr ? min(*p.todo_count, c.P) : c.P;
-    for (int32_t it = blockIdx.x * wpb + warp; it < count; it += gridDim.x * wpb) {
-        const int32_t b = p.todo != nullptr ? p.todo[it] : it;
-        const int32_t T = p.lens[b];
+    // the parent after this one is looked up while this one is evaluated (index, then length and row offset)
+    const int32_t it_step = gridDim.x * wpb;
+    int32_t it = blockIdx.x * wpb + warp;
+    int32_t b_nx = it < count ? (p.todo != nullptr ? p.todo[it] : it) : 0;
+    int32_t T_nx = it < count ? p.lens[b_nx] : 0;
+    int64_t off_nx = it < count ? p.offs[b_nx] : 0;
+    for (; it < count; it += it_step) {
+        const int32_t b = b_nx, T = T_nx;
+        const int64_t off = off_nx;
+        const bool more = it + it_step < count;
+        b_nx = more ? (p.todo != nullptr ? p.todo[it + it_step] : it + it_step) : 0;
+        bool got_nx = false;
         int64_t out_pk = -1, out_du = -1;
         int32_t out_st = -2;
         uint16_t* row = c.row + (int64_t)b * c.stride16;
@@ -166,7 +175,7 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
             for (int32_t i = lane; i < c.stride + 4; i += 32) arrA[i] = 0;
             __syncwarp();
             // ---- occurrence words (1-based steps, 16 bits each) and the copy of the row
-            const int32_t* src = p.seqs + p.offs[b];
+            const int32_t* src = p.seqs + off;
             auto put = [&](int32_t v, int32_t t) {
                 row[t] = (uint16_t)v;
                 const uint32_t slot = min((uint32_t)v, (uint32_t)n);      // ids outside [0, n) land in a spare word
@@ -183,6 +192,7 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
                     if (t0 + 32 * k < T) put(v[k], t0 + 32 * k);
             }
             __syncwarp();
+            if (more) { T_nx = p.lens[b_nx]; off_nx = p.offs[b_nx]; got_nx = true; }
             // ---- per node: both copies a <= b, free steps from the successors' copies, profile deltas
             uint32_t vsum = 0;
             bool absent = false, dep = false, over = false;
@@ -370,6 +380,7 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
             }
             __syncwarp();
         }
+        if (more && !got_nx) { T_nx = p.lens[b_nx]; off_nx = p.offs[b_nx]; }
         if (lane == 0) {
             c.len[b] = T;
             c.status[b] = out_st;
