@@ -121,9 +121,9 @@ __device__ __forceinline__ void edit_add(int64_t* p, int64_t v) {
 // (sequence length, for sinks) and, at the next multiple of four after n + 2, the constant word of empty node slots.
 __host__ __device__ inline int32_t edit_word_stride(int32_t n) { return ((n + 2 + 3) & ~3) + 4; }
 
-// Shared memory of one warp: occurrence words [edit_word_stride(n)] uint32, then two arrays of stride + 4 MemT.
+// Shared memory of one warp (cache build): occurrence words [edit_word_stride(n)] uint32, then two arrays of stride + 8 MemT.
 __host__ __device__ inline size_t edit_warp_bytes(int32_t n, int32_t stride, size_t mem_sz) {
-    return (size_t)edit_word_stride(n) * 4 + 2 * ((((size_t)stride + 4) * mem_sz + 15) & ~size_t(15));
+    return (size_t)edit_word_stride(n) * 4 + 2 * ((((size_t)stride + 8) * mem_sz + 15) & ~size_t(15));
 }
 
 // Full evaluation of every parent (same quantities as the evaluation kernels: Section 2, Eqs. 1-8)
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
     }
     char* ws = smem + (kChip ? p.chip_bytes : 0u) + (size_t)warp * p.warp_bytes;
     uint32_t* word = reinterpret_cast<uint32_t*>(ws);
-    const size_t arr_bytes = (((size_t)c.stride + 4) * sizeof(MemT) + 15) & ~size_t(15);
+    const size_t arr_bytes = (((size_t)c.stride + 8) * sizeof(MemT) + 15) & ~size_t(15);
     const int32_t n = c.n, wstride = edit_word_stride(c.n);
     MemT* arrA = reinterpret_cast<MemT*>(ws + (size_t)wstride * 4);
     MemT* arrB = reinterpret_cast<MemT*>(ws + (size_t)wstride * 4 + arr_bytes);
@@ -171,8 +171,8 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
         int32_t out_st = -2;
         uint16_t* row = c.row + (int64_t)b * c.stride16;
         if (T >= n && T <= c.max_T) {
-            for (int32_t i = lane; i < wstride; i += 32) word[i] = 0;
-            for (int32_t i = lane; i < c.stride + 4; i += 32) arrA[i] = 0;
+            for (int32_t i = lane; i < wstride / 4; i += 32) reinterpret_cast<uint4*>(word)[i] = make_uint4(0, 0, 0, 0);
+            for (int32_t i = lane; i < (int32_t)arr_bytes / 16; i += 32) reinterpret_cast<uint4*>(arrA)[i] = make_uint4(0, 0, 0, 0);
             __syncwarp();
             // ---- occurrence words (1-based steps, 16 bits each) and the copy of the row
             const int32_t* src = p.seqs + off;
@@ -288,7 +288,12 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
                 over = __any_sync(kFull, (int32_t)capw < 0) || (int)((acc_all >> kPairCntShift) & 0x7FFFu) != T - n;
                 dep = (depw & 0x80008000u) != 0;
                 __syncwarp();
-                for (int32_t t = lane; t < T; t += 32) fre[t] = (uint16_t)arrB[t];
+                for (int32_t t = 8 * lane; t < T; t += 256) {             // eight free steps per 16-byte store
+                    uint32_t q[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) q[i] = ((uint32_t)arrB[t + 2 * i] & 0xFFFFu) | (uint32_t)arrB[t + 2 * i + 1] << 16;
+                    *reinterpret_cast<uint4*>(fre + t) = make_uint4(q[0], q[1], q[2], q[3]);
+                }
                 // position sum and duration in the form the rest of the kernel expects
                 vsum = lane == 0 ? (uint32_t)T * ((uint32_t)T + 1u) / 2u : 0u;
                 dur = lane == 0 ? p.base_dur + (int64_t)(acc_all & kPairDurMask) : 0;
@@ -334,46 +339,70 @@ __global__ void __launch_bounds__(kPrepThreads) edit_prepare_kernel(const PrepPa
                 out_st = -1;
                 out_du = dur;
             } else if (well) {
-                // ---- profile, prefix maxima, suffix maxima: lane owns a run of consecutive steps
-                const int32_t per = ((T + 31) / 32) | 1;                  // odd: the lanes' runs start in different banks
-                const int32_t t0 = min(T, lane * per), t1 = min(T, t0 + per);
-                MemT sum = 0;
-                for (int32_t t = t0; t < t1; ++t) sum += arrA[t];
-                MemT run = edit_warp_incl_sum(sum, lane) - sum;
-                MemT top = 0;
-                for (int32_t t = t0; t < t1; ++t) {
-                    run += arrA[t];
-                    arrA[t] = run;                                          // prof
-                    top = run > top ? run : top;
+                // ---- profile, prefix maxima, suffix maxima: lane owns a run of consecutive steps, a whole number
+                // of 16-byte vectors long and an odd number of them (the lanes' vectors fall into different banks).
+                // Steps T .. Tp - 1 pad the last vector: their deltas are 0 and the usage there is 0.
+                constexpr int32_t VW = 16 / (int32_t)sizeof(MemT);
+                const int32_t Tp = (T + VW - 1) & ~(VW - 1);
+                const int32_t per = VW * ((((T + 31) / 32 + VW - 1) / VW) | 1);
+                const int32_t t0 = min(Tp, lane * per), t1 = min(Tp, t0 + per);
+                auto ldv = [](const MemT* a, MemT (&v)[VW]) { *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(a); };
+                auto stv = [](MemT* a, const MemT (&v)[VW]) { *reinterpret_cast<uint4*>(a) = *reinterpret_cast<const uint4*>(v); };
+                // pass 1: sum and largest running sum of the run, both relative to its start
+                MemT sum = 0, top = 0;
+                for (int32_t t = t0; t < t1; t += VW) {
+                    alignas(16) MemT v[VW];
+                    ldv(arrA + t, v);
+#pragma unroll
+                    for (int i = 0; i < VW; ++i) { sum += v[i]; top = sum > top ? sum : top; }
                 }
+                MemT run = edit_warp_incl_sum(sum, lane) - sum;             // usage in front of the run
+                top += run;                                                 // largest usage inside the run (0 for an empty one)
                 MemT carry = edit_warp_incl_max_up(top, lane);
                 const MemT peak = __shfl_sync(kFull, carry, 31);
                 carry = __shfl_up_sync(kFull, carry, 1);
                 if (lane == 0) carry = 0;
-                for (int32_t t = t0; t < t1; ++t) {
-                    carry = arrA[t] > carry ? arrA[t] : carry;
-                    arrB[t] = carry;                                        // pm
+                // pass 2: usage and prefix maxima
+                for (int32_t t = t0; t < t1; t += VW) {
+                    alignas(16) MemT v[VW], w[VW];
+                    ldv(arrA + t, v);
+#pragma unroll
+                    for (int i = 0; i < VW; ++i) {
+                        run += v[i];
+                        v[i] = run;
+                        carry = run > carry ? run : carry;
+                        w[i] = carry;
+                    }
+                    stv(arrA + t, v);                                       // prof
+                    stv(arrB + t, w);                                       // pm
                 }
                 __syncwarp();
-                MemT* g_prof = reinterpret_cast<MemT*>(c.prof) + (int64_t)b * c.stride;
-                MemT* g_pm = reinterpret_cast<MemT*>(c.pm) + (int64_t)b * c.stride;
-                MemT* g_sm = reinterpret_cast<MemT*>(c.sm) + (int64_t)b * c.stride;
-                for (int32_t t = lane; t < T; t += 32) {
-                    g_prof[t] = arrA[t];
-                    g_pm[t] = arrB[t];
+                uint4* g_prof = reinterpret_cast<uint4*>(reinterpret_cast<MemT*>(c.prof) + (int64_t)b * c.stride);
+                uint4* g_pm = reinterpret_cast<uint4*>(reinterpret_cast<MemT*>(c.pm) + (int64_t)b * c.stride);
+                uint4* g_sm = reinterpret_cast<uint4*>(reinterpret_cast<MemT*>(c.sm) + (int64_t)b * c.stride);
+                for (int32_t i = lane; i < Tp / VW; i += 32) {
+                    g_prof[i] = reinterpret_cast<const uint4*>(arrA)[i];
+                    g_pm[i] = reinterpret_cast<const uint4*>(arrB)[i];
                 }
                 __syncwarp();
+                // pass 3: suffix maxima
                 MemT back = edit_warp_incl_max_down(top, lane);
                 back = __shfl_down_sync(kFull, back, 1);
                 if (lane == 31) back = 0;
-                for (int32_t t = t1 - 1; t >= t0; --t) {
-                    back = arrA[t] > back ? arrA[t] : back;
-                    arrB[t] = back;                                         // sm
+                for (int32_t t = t1 - VW; t >= t0; t -= VW) {
+                    alignas(16) MemT v[VW], w[VW];
+                    ldv(arrA + t, v);
+#pragma unroll
+                    for (int i = VW - 1; i >= 0; --i) {
+                        back = v[i] > back ? v[i] : back;
+                        w[i] = back;
+                    }
+                    stv(arrB + t, w);                                       // sm
                 }
                 __syncwarp();
-                for (int32_t t = lane; t < T; t += 32) g_sm[t] = arrB[t];
-                uint32_t* g_occ = c.occ + (int64_t)b * c.occ_stride;
-                for (int32_t u = lane; u < n; u += 32) g_occ[u] = word[u];
+                for (int32_t i = lane; i < Tp / VW; i += 32) g_sm[i] = reinterpret_cast<const uint4*>(arrB)[i];
+                uint4* g_occ = reinterpret_cast<uint4*>(c.occ + (int64_t)b * c.occ_stride);
+                for (int32_t i = lane; i < c.occ_stride / 4; i += 32) g_occ[i] = reinterpret_cast<const uint4*>(word)[i];
                 out_pk = (int64_t)peak;
                 out_du = dur;
                 out_st = out_pk <= p.M ? 1 : 0;
