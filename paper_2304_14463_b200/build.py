@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoc_b200.so")
 SOURCES = ["moc_api.cu", "moc_search.cu", "moc_intervals.cu", "moc_edits.cu"]
-HEADERS = ["moc_kernels.cuh", "moc_pair_kernel.cuh", "moc_lane_kernel.cuh", "moc_quad_kernel.cuh", "moc_host.cuh", "moc_search_kernels.cuh", "moc_search_score_kernel.cuh", "moc_interval_kernels.cuh", "moc_edit_kernels.cuh", "moc_cache_host.cuh", os.path.join("..", "..", "include", "moc.h")]
+HEADERS = ["moc_kernels.cuh", "moc_pair_kernel.cuh", "moc_lane_kernel.cuh", "moc_quad_kernel.cuh", "moc_host.cuh", "moc_search_kernels.cuh", "moc_search_score_kernel.cuh", "moc_edit_pass.cuh", "moc_edit_lanes_kernel.cuh", "moc_interval_kernels.cuh", "moc_edit_kernels.cuh", "moc_cache_host.cuh", os.path.join("..", "..", "include", "moc.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "--use_fast_math"]
 

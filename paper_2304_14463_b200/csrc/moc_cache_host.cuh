@@ -2,6 +2,7 @@
 #pragma once
 #include "moc_host.cuh"
 #include "moc_edit_kernels.cuh"
+#include "moc_edit_lanes_kernel.cuh"
 
 struct moc_cache {
     const moc_graph* g = nullptr;
@@ -14,6 +15,12 @@ struct moc_cache {
     moc::EditCacheDev c{};
     size_t warp_bytes = 0;
     int wpb = 0, grid_cap = 0;
+    // launch of the lane-per-edit kernel, made on the first moc_eval_edits (0: not yet, -1: the graph does not fit it)
+    mutable int lanes_state = 0;
+    mutable moc::LanesParams lanes{};
+    mutable const void* lanes_fn = nullptr;
+    mutable size_t lanes_smem = 0;
+    mutable int lanes_grid_cap = 0;
 };
 
 namespace moc_host {

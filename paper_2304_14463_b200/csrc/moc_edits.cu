@@ -187,6 +187,46 @@ int moc_eval_edits(const moc_cache* h, const int32_t* parent, const int32_t* op,
     p.out_status = out_status;
     p.out_window = out_window;
     const size_t msz = h->wide ? 8 : 4;
+    const moc_graph* g = h->g;
+    // ---- a lane per edit, when the correction lists of a warp and (if it fits) the graph find room on an SM
+    if (h->lanes_state == 0) {
+        h->lanes_state = -1;
+        moc::LanesParams& lp = h->lanes;
+        lp.list_cap = std::max(128, (4 + 2 * g->max_indeg + 31) & ~31);
+        lp.warp_bytes = (uint32_t)moc::lanes_warp_bytes(h->c.stride, msz, lp.list_cap, &lp.lh_b, &lp.diff_b);
+        const size_t cap = g->smem_optin > 2048 ? g->smem_optin - 2048 : 0;
+        const int wpb = moc::kLanesThreads / 32;
+        const size_t graph_b = moc::score_graph_bytes(g->n, g->n_edges, msz, &lp.gs_pred_b, &lp.gs_m_b, &lp.gs_succ_b, &lp.gs_predl_b);
+        for (int chip = 1; chip >= 0 && h->lanes_state < 0; --chip) {
+            if (chip && (g->n > 65535 || graph_b > cap / 8)) continue;
+            const size_t smem = (chip ? graph_b : 0) + (size_t)lp.warp_bytes * wpb;
+            if (smem > cap) continue;
+            const void* fn = chip ? (h->wide ? (const void*)moc::edit_eval_lanes_kernel<int64_t, true> : (const void*)moc::edit_eval_lanes_kernel<int32_t, true>)
+                                  : (h->wide ? (const void*)moc::edit_eval_lanes_kernel<int64_t, false> : (const void*)moc::edit_eval_lanes_kernel<int32_t, false>);
+            MOC_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(g->smem_optin - 1024)));
+            int nb = 0;
+            MOC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, moc::kLanesThreads, smem));
+            if (nb < 1) continue;
+            lp.graph_bytes = chip ? (uint32_t)graph_b : 0u;
+            h->lanes_fn = fn;
+            h->lanes_smem = smem;
+            h->lanes_grid_cap = g->sm_count * nb;
+            h->lanes_state = 1;
+        }
+    }
+    if (h->lanes_state > 0) {
+        moc::LanesParams lp = h->lanes;
+        lp.e = p;
+        lp.e.c.cap = g->d_cap;
+        const int wpb = moc::kLanesThreads / 32;
+        const int64_t n_groups = ((int64_t)B + 31) / 32;
+        const int grid = (int)std::min<int64_t>(h->lanes_grid_cap, (n_groups + wpb - 1) / wpb);
+        void* args[] = {&lp};
+        MOC_CUDA(cudaLaunchKernel(h->lanes_fn, dim3(grid), dim3(moc::kLanesThreads), args, h->lanes_smem, (cudaStream_t)stream));
+        launch_counter() = 1;
+        return MOC_OK;
+    }
+    // ---- a warp per edit
     const size_t warp_b = 2 * ((((size_t)h->c.stride + 4) * msz + 15) & ~size_t(15));
     p.warp_bytes = (uint32_t)warp_b;
     const int wpb = moc::kEditThreads / 32;

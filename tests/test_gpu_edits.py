@@ -59,9 +59,16 @@ def run_case(B, wl, seqs, lens, M, parent, op, q, j, caps=None, what=""):
     torch.cuda.synchronize()
     rp, rd, rs, _ = O.eval_batch(seqs, lens, M)
     assert (pk.cpu().numpy() == rp).all() and (du.cpu().numpy() == rd).all() and (st.cpu().numpy() == rs).all(), what
-    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    window = torch.full((len(parent),), -7, dtype=torch.int32, device="cuda")
+    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M, window=window)
     torch.cuda.synchronize()
     got = np.stack([got[0].cpu().numpy(), got[1].cpu().numpy(), got[2].cpu().numpy().astype(np.int64)], 1)
+    # steps whose usage was recomputed: none for a refused edit, at most the child's length for a scored one
+    win = window.cpu().numpy()
+    scored = got[:, 2] >= 0
+    child_len = lens[np.clip(parent, 0, len(lens) - 1)] + (op == 0) - (op == 1)
+    assert (win[~scored] == 0).all() and (win[scored] >= 0).all() and (win[scored] <= child_len[scored]).all(), what
+    assert not scored.any() or win[scored].max() > 0, what
     want = reference(O, seqs, lens, parent, op, q, j, M, rs)
     bad = np.nonzero((got != want).any(1))[0]
     assert len(bad) == 0, f"{what}: {len(bad)} of {len(parent)} edits differ; first: edit {bad[0]} parent {parent[bad[0]]} " \
@@ -177,9 +184,16 @@ def test_stale_cache_is_refused(B):
     G.set_caps(caps)
     O.set_caps(caps)
     cache.build(dev(seqs), dev(lens), M)
-    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M)
+    window = torch.full((len(parent),), -7, dtype=torch.int32, device="cuda")
+    got = cache.eval_edits(dev(parent), dev(op), dev(q), dev(j), M, window=window)
     torch.cuda.synchronize()
     got = np.stack([got[0].cpu().numpy(), got[1].cpu().numpy(), got[2].cpu().numpy().astype(np.int64)], 1)
+    # steps whose usage was recomputed: none for a refused edit, at most the child's length for a scored one
+    win = window.cpu().numpy()
+    scored = got[:, 2] >= 0
+    child_len = lens[np.clip(parent, 0, len(lens) - 1)] + (op == 0) - (op == 1)
+    assert (win[~scored] == 0).all() and (win[scored] >= 0).all() and (win[scored] <= child_len[scored]).all(), what
+    assert not scored.any() or win[scored].max() > 0, what
     want = reference(O, seqs, lens, parent, op, q, j, M, O.eval_batch(seqs, lens, M)[2])
     assert (got == want).all()
     torch.cuda.synchronize()
