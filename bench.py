@@ -462,8 +462,8 @@ def run_edits(args):
             "status_counts": {str(k): int((st == k).sum()) for k in (1, 0, -1, -2, -3)},
             "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
                          "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak_gbs, "peak_kind": f"of {peak_kind}",
-                         "traffic": 104447232 + 4538112,
-                         "traffic_source": "ncu, one launch of this workload: dram read 104.45 MB, write 4.54 MB",
+                         "traffic": 101489664 + 3884544,
+                         "traffic_source": "ncu, one launch of this workload (edit_eval_lanes_kernel): dram read 101.49 MB, write 3.88 MB",
                          "algorithmic_bytes_per_launch": alg_bytes},
             "clocks": clocks.summary()}
     if not args.no_cpu_baseline:

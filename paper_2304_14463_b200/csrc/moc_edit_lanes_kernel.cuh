@@ -56,7 +56,7 @@ struct LaneParent {
 };
 
 template <typename MemT, bool kGraphOnChip>
-__global__ void __launch_bounds__(kLanesThreads) edit_eval_lanes_kernel(const LanesParams p) {
+__global__ void __launch_bounds__(kLanesThreads, 4) edit_eval_lanes_kernel(const LanesParams p) {
     extern __shared__ __align__(16) char smem[];
     const EditParams& e = p.e;
     const EditCacheDev& c = e.c;
