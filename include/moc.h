@@ -362,8 +362,8 @@ int moc_search_set_kinds(moc_search* s, uint32_t kinds);
  *                (E must be 1);
  *                1 (MOC_SEARCH_SCORE_AUTO): proposals are scored from the cached evaluation of the chain's
  *                sequence and only accepted ones are written out; the library picks the scoring kernel
- *                (a warp per chain from E = 2 on when the graph fits it, else a warp per proposal);
- *                2 (MOC_SEARCH_SCORE_EDIT): the same with a warp per proposal: a generation is four
+ *                (a warp per chain from E = 24 on when the graph fits it, else the kernel of moc_eval_edits);
+ *                2 (MOC_SEARCH_SCORE_EDIT): the same through moc_eval_edits: a generation is four
  *                kernels (draw, moc_eval_edits, pick, rebuild of the changed cache entries);
  *                3 (MOC_SEARCH_SCORE_CHAIN): the same with a warp per chain: the chain's cache entry is
  *                staged in shared memory once and its E proposals are drawn, scored and settled there;

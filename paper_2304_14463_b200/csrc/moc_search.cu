@@ -316,9 +316,10 @@ int moc_search_set_samples(moc_search* s, int32_t samples, int32_t incremental) 
     ip.todo = (int32_t*)(b + o_todo);
     ip.todo_count = (int32_t*)(b + o_cnt);
     MOC_CUDA(cudaMemset(ip.todo_count, 0, 8));
-    // scoring kernel: a warp per chain when asked for, or by default from two proposals per chain on
+    // scoring kernel: a warp per chain when asked for, or by default from 24 proposals per chain on
+    // (below that the lane-per-edit kernel of moc_eval_edits, with more warps per SM, is as fast or faster)
     s->fused = false;
-    if (incremental == MOC_SEARCH_SCORE_CHAIN || (incremental == MOC_SEARCH_SCORE_AUTO && samples >= 2)) {
+    if (incremental == MOC_SEARCH_SCORE_CHAIN || (incremental == MOC_SEARCH_SCORE_AUTO && samples >= 24)) {
         s->fused = plan_fused(s);
         if (!s->fused && incremental == MOC_SEARCH_SCORE_CHAIN) {
             cudaFree(s->d_inc);
