@@ -158,6 +158,32 @@ def test_edits_node_caps_and_wide(B):
     run_case(B, wl, seqs, lens, M * (1 << 33), *random_edits(rng, lens, 4000), what="wide")
 
 
+def test_edits_of_a_star_graph(B):
+    """In-degree 1199: the correction lists of the lane-per-edit kernel (4 + 2 * in-degree entries per edit) do not
+    fit eight warps of an SM, so the warp-per-edit kernel scores; same results."""
+    class WL:
+        pass
+    wl = WL()
+    n = 1200
+    rng = np.random.default_rng(21)
+    wl.n, wl.C = n, 2
+    wl.edges = np.array([(i, n - 1) for i in range(n - 1)], np.int32)
+    wl.w = rng.integers(1, 9, n).astype(np.int64)
+    wl.m = rng.integers(1, 99, n).astype(np.int64)
+    rows = []
+    for _ in range(8):
+        r = list(rng.permutation(n - 1)) + [n - 1]
+        for v in rng.integers(0, n - 1, 40):                       # a second copy of some sources, in front of the sink
+            if r.count(int(v)) == 1:
+                r.insert(int(rng.integers(r.index(int(v)) + 1, len(r))), int(v))
+        rows.append(r)
+    seqs = np.array([x for r in rows for x in r], np.int32)
+    lens = np.array([len(r) for r in rows], np.int32)
+    M = int(wl.m.sum()) * 9 // 10
+    want = run_case(B, wl, seqs, lens, M, *random_edits(rng, lens, 3000), what="star")
+    assert {0, -1, -2} <= set(want[:, 2].tolist()) or {1, -1, -2} <= set(want[:, 2].tolist())
+
+
 def test_stale_cache_is_refused(B):
     """Caps or C changed after the build: the cache's copy is stale, edits are refused until a rebuild,
     and after the rebuild they follow the new caps."""
