@@ -57,10 +57,11 @@ bool plan_fused(moc_search* s) {
     if ((size_t)sp.warp_bytes * 4 > cap) return false;
     // with the block's own copy of the graph when that still leaves eight warps on an SM, else from global memory
     const int64_t E = g->n_edges;
-    sp.graph_bytes = (uint32_t)moc::score_graph_bytes(g->n, E, msz, &sp.gs_pred_b, &sp.gs_m_b, &sp.gs_succ_b, &sp.gs_predl_b);
+    const size_t graph_b = moc::score_graph_bytes(g->n, E, msz, &sp.gs_pred_b, &sp.gs_m_b, &sp.gs_succ_b, &sp.gs_predl_b);
+    sp.graph_bytes = (uint32_t)std::min<size_t>(graph_b, 0xFFFFFFF0u);
     int best = 0;
     for (int chip = 1; chip >= 0; --chip) {
-        if (chip && (g->n > 65535 || sp.graph_bytes > cap / 4)) continue;
+        if (chip && (g->n > 65535 || graph_b > cap / 4)) continue;
         s->score_fn = chip ? (h->wide ? (const void*)moc::search_score_kernel<int64_t, true> : (const void*)moc::search_score_kernel<int32_t, true>)
                            : (h->wide ? (const void*)moc::search_score_kernel<int64_t, false> : (const void*)moc::search_score_kernel<int32_t, false>);
         if (cudaFuncSetAttribute(s->score_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(g->smem_optin - 1024)) != cudaSuccess) {
