@@ -41,6 +41,7 @@ struct IntervalParams {
     int32_t* out_lens;           // B, or nullptr
     uint32_t words;              // bitmap words: (D + 32) / 32  (bit t of the bitmap = event t, bit 0 unused)
     uint32_t warp_bytes;         // shared memory of one warp
+    int32_t byte_marks;          // plain model, and two bytes per event fit the space of the difference array
 };
 
 // Shared memory of one warp, in this order: bitmap of active starts [words], bitmap of all starts
@@ -87,6 +88,11 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
     MemT* delta = reinterpret_cast<MemT*>(ws + interval_bitmap_bytes(p.words, kPlain));
     PosT* sS = reinterpret_cast<PosT*>(ws + interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)));
     PosT* sE = sS + K;
+    // plain model: one byte per event and kind of mark (active starts, all starts) during pass 1, in the space of
+    // the difference array (2 (D + 1) <= (K + 2) sizeof(MemT) since D = K there)
+    const uint32_t by_stride = ((uint32_t)p.D + 1u + 15u) & ~15u;
+    uint8_t* by_act = reinterpret_cast<uint8_t*>(delta);
+    uint8_t* by_all = by_act + by_stride;
     constexpr uint32_t kFull = 0xFFFFFFFFu;
     const int nz = (int)(interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)) >> 4);
 
@@ -135,19 +141,23 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                         sE[v * C + i] = (PosT)ev[i];
                     }
                     if (in_dom) {
+                        // Each node marks its distinct starts; Eq. 6 holds iff no two nodes marked the same event,
+                        // i.e. iff as many events end up marked as marks were made.  With byte marks (plain
+                        // stores: marks of neighbouring events share a word without colliding) the two bitmaps
+                        // are made from the bytes below; otherwise the marks go straight into them.
                         const uint32_t bit = 1u << (sv[i] & 31);
                         if (act) {
-                            atomicOr(&bm_act[sv[i] >> 5], bit);
+                            if (kPlain && p.byte_marks) by_act[sv[i]] = 1;
+                            else atomicOr(&bm_act[sv[i] >> 5], bit);
                             if (!kPlain && !((int64_t)sv[i] >= k && is_triangular_from((int64_t)sv[i] - k, k))) mask |= kIvStage;
                         }
                         if (kPlain) {
-                            // each node marks its distinct starts; Eq. 6 holds iff no two nodes marked the same
-                            // bit, i.e. iff the bitmap ends up with as many bits as marks were made
                             bool seen = false;
 #pragma unroll
                             for (int i2 = 0; i2 < i; ++i2) seen |= sv[i2] == sv[i];
                             if (!seen) {
-                                atomicOr(&bm_all[sv[i] >> 5], bit);
+                                if (p.byte_marks) by_all[sv[i]] = 1;
+                                else atomicOr(&bm_all[sv[i] >> 5], bit);
                                 ++n_distinct;
                             }
                         }
@@ -166,6 +176,23 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
             continue;
         }
         __syncwarp();
+        if (kPlain && p.byte_marks) {
+            // bytes -> bitmaps: the warp reads 32 consecutive events, the ballot is their bitmap word; then the
+            // bytes, which borrowed the difference array, are cleared again
+            for (uint32_t wd = 0; wd < p.words; ++wd) {
+                const int32_t t = (int32_t)(wd * 32u) + lane;
+                const bool in = t <= p.D;
+                const uint32_t ba = __ballot_sync(kFull, in && by_act[t] != 0), bl = __ballot_sync(kFull, in && by_all[t] != 0);
+                if (lane == 0) {
+                    bm_act[wd] = ba;
+                    bm_all[wd] = bl;
+                }
+            }
+            __syncwarp();
+            int4* z4 = reinterpret_cast<int4*>(by_act);
+            for (uint32_t i = lane; i < (2u * by_stride + 15u) / 16u; i += 32) z4[i] = make_int4(0, 0, 0, 0);
+            __syncwarp();
+        }
 
         // ---- rank base of every bitmap word: exclusive prefix sum of the popcounts
         int32_t R;

@@ -51,6 +51,7 @@ extern "C" int moc_check_intervals(const moc_graph* g, const int32_t* s, const i
         return fail(MOC_ERR_ARG, "moc_check_intervals: domain of %lld events with %lld intervals needs %zu bytes of "
                     "shared memory per solution, the device offers %zu", (long long)D, (long long)K, base_b, cap);
     // keep the solution on chip after the first pass while at least eight solutions per SM still fit
+    p.byte_marks = plain && 2 * (((size_t)D + 1 + 15) & ~size_t(15)) <= ((((size_t)K + 2) * (wide ? 8 : 4) + 15) & ~size_t(15)) ? 1 : 0;
     const bool stage = (base_b + stage_b) * 8 <= cap;
     const size_t warp_b = base_b + (stage ? stage_b : 0);
     p.warp_bytes = (uint32_t)warp_b;
