@@ -261,17 +261,29 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                     ue[j] = 0;
                 }
             }
+            // Eq. 5: every active start t of a successor lies in (us, ue] of one slot of u, tested as
+            // (t - lo) <= len in unsigned arithmetic with lo = us + 1, len = ue - lo; a slot that serves nobody
+            // (inactive, or ue <= us) gets lo = 2^32 - 1, len = 0, which no t >= 1 satisfies
+            uint32_t lo5[CP], len5[CP];
+#pragma unroll
+            for (int j = 0; j < CP; ++j) {
+                const bool serves = ue[j] > us[j];
+                lo5[j] = serves ? (uint32_t)us[j] + 1u : 0xFFFFFFFFu;
+                len5[j] = serves ? (uint32_t)(ue[j] - us[j] - 1) : 0u;
+            }
             const int32_t e0 = __ldg(&p.succ_start[u]), e1 = __ldg(&p.succ_start[u + 1]);
             for (int32_t q = e0; q < e1; ++q) {
                 const int32_t v = __ldg(&p.succ[q]);
-                for (int32_t i = 0; i < C; ++i) {
-                    int32_t t, te;
-                    slot(v, i, t, te);
-                    if (t == 0) continue;
-                    bool found = false;
 #pragma unroll
-                    for (int j = 0; j < CP; ++j) found |= us[j] + 1 <= t && t <= ue[j];
-                    if (!found) mask |= kIvEq5;
+                for (int i = 0; i < CP; ++i) {
+                    if (i < C) {
+                        int32_t t, te;
+                        slot(v, i, t, te);
+                        bool found = t == 0;                    // an inactive slot of the successor asks for nothing
+#pragma unroll
+                        for (int j = 0; j < CP; ++j) found |= (uint32_t)t - lo5[j] <= len5[j];
+                        if (!found) mask |= kIvEq5;
+                    }
                 }
             }
         }
