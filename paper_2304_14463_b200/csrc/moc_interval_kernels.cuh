@@ -105,6 +105,8 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
             for (int i = lane; i < nz; i += 32) z4[i] = make_int4(0, 0, 0, 0);
         }
         __syncwarp();
+        // C = 2 and the three rows of this solution start on 8 bytes: slots are read in pairs
+        const bool pairs = C == 2 && ((reinterpret_cast<uintptr_t>(gs) | reinterpret_cast<uintptr_t>(ge) | reinterpret_cast<uintptr_t>(ga)) & 7) == 0;
 
         // ---- pass 1, per node: read the C slots; Eq. 8; Eqs. 1, 2, 3, 7; mark the starts in the bitmaps
         // (Eq. 6 / staged rule).  A start outside the domain marks nothing; the marks are used only when
@@ -113,12 +115,20 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         int64_t dur = 0;
         for (int32_t v = lane; v < n; v += 32) {
             int32_t sv[CP], ev[CP], av[CP];
+            if (CP == 2 && pairs) {                         // two slots per node: one 8-byte load per array
+                const int2 s2 = __ldg(reinterpret_cast<const int2*>(gs) + v), e2 = __ldg(reinterpret_cast<const int2*>(ge) + v),
+                           a2 = __ldg(reinterpret_cast<const int2*>(ga) + v);
+                sv[0] = s2.x; sv[1] = s2.y;
+                ev[0] = e2.x; ev[1] = e2.y;
+                av[0] = a2.x; av[1] = a2.y;
+            } else {
 #pragma unroll
-            for (int i = 0; i < CP; ++i) {
-                const bool in = i < C;
-                sv[i] = in ? __ldg(gs + v * C + i) : 0;
-                ev[i] = in ? __ldg(ge + v * C + i) : 0;
-                av[i] = in ? __ldg(ga + v * C + i) : 0;
+                for (int i = 0; i < CP; ++i) {
+                    const bool in = i < C;
+                    sv[i] = in ? __ldg(gs + v * C + i) : 0;
+                    ev[i] = in ? __ldg(ge + v * C + i) : 0;
+                    av[i] = in ? __ldg(ga + v * C + i) : 0;
+                }
             }
             const int64_t wv = __ldg(&p.w[v]);
             int64_t k = 0;
@@ -127,6 +137,10 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                 if ((int64_t)sv[0] != k * (k + 1) / 2) mask |= kIvStage;
             }
             if (av[0] != 1) mask |= kIvEq7;
+            if (kStage && CP == 2 && sizeof(PosT) == 2 && C == 2) {       // both slots in one 32-bit store per array
+                reinterpret_cast<uint32_t*>(sS)[v] = (uint32_t)(uint16_t)(av[0] == 1 ? sv[0] : 0) | (uint32_t)(uint16_t)(av[1] == 1 ? sv[1] : 0) << 16;
+                reinterpret_cast<uint32_t*>(sE)[v] = (uint32_t)(uint16_t)ev[0] | (uint32_t)(uint16_t)ev[1] << 16;
+            }
 #pragma unroll
             for (int i = 0; i < CP; ++i) {
                 if (i < C) {
@@ -136,7 +150,7 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                     if (i + 1 < CP && i + 1 < C && ev[i] > sv[i + 1]) mask |= kIvEq3;
                     const bool act = av[i] == 1;
                     if (act) { dur += wv; ++n_act; }
-                    if (kStage) {
+                    if (kStage && !(CP == 2 && sizeof(PosT) == 2 && C == 2)) {
                         sS[v * C + i] = (PosT)(act ? sv[i] : 0);
                         sE[v * C + i] = (PosT)ev[i];
                     }
@@ -229,6 +243,10 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
             return (int32_t)(rbase[t >> 5] + __popc(wd & (0xFFFFFFFFu >> (31 - (t & 31)))));
         };
         // start (0 = inactive) and end of slot i of node v
+        // both slots of node v at once (C = 2, positions staged in 16 bits)
+        constexpr bool kPairStage = kStage && CP == 2 && sizeof(PosT) == 2;
+        auto start_pair = [&](int32_t v) -> uint32_t { return reinterpret_cast<const uint32_t*>(sS)[v]; };
+        auto end_pair = [&](int32_t v) -> uint32_t { return reinterpret_cast<const uint32_t*>(sE)[v]; };
         auto slot = [&](int32_t v, int32_t i, int32_t& s_out, int32_t& e_out) {
             if (kStage) {
                 s_out = (int32_t)sS[v * C + i];
@@ -244,11 +262,20 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         for (int32_t u = lane; u < n; u += 32) {
             int32_t us[CP], ue[CP];
             const MemT mv = (MemT)__ldg(&p.m[u]);
+            if (kPairStage && C == 2) {
+                const uint32_t sp = start_pair(u), ep = end_pair(u);
+                us[0] = (int32_t)(sp & 0xFFFFu); us[1] = (int32_t)(sp >> 16);
+                ue[0] = (int32_t)(ep & 0xFFFFu); ue[1] = (int32_t)(ep >> 16);
+            } else {
+#pragma unroll
+                for (int j = 0; j < CP; ++j) {
+                    us[j] = 0;
+                    ue[j] = 0;
+                    if (j < C) slot(u, j, us[j], ue[j]);
+                }
+            }
 #pragma unroll
             for (int j = 0; j < CP; ++j) {
-                us[j] = 0;
-                ue[j] = 0;
-                if (j < C) slot(u, j, us[j], ue[j]);
                 if (us[j] != 0) {
                     const int32_t r = rank(us[j]);
                     if (us[j] <= ue[j]) {
@@ -274,11 +301,14 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
             const int32_t e0 = __ldg(&p.succ_start[u]), e1 = __ldg(&p.succ_start[u + 1]);
             for (int32_t q = e0; q < e1; ++q) {
                 const int32_t v = __ldg(&p.succ[q]);
+                uint32_t tp = 0;
+                if (kPairStage && C == 2) tp = start_pair(v);
 #pragma unroll
                 for (int i = 0; i < CP; ++i) {
                     if (i < C) {
-                        int32_t t, te;
-                        slot(v, i, t, te);
+                        int32_t t, te = 0;
+                        if (kPairStage && C == 2) t = (int32_t)(i == 0 ? tp & 0xFFFFu : tp >> 16);
+                        else slot(v, i, t, te);
                         bool found = t == 0;                    // an inactive slot of the successor asks for nothing
 #pragma unroll
                         for (int j = 0; j < CP; ++j) found |= (uint32_t)t - lo5[j] <= len5[j];
