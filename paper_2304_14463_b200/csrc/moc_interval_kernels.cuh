@@ -88,11 +88,10 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
     MemT* delta = reinterpret_cast<MemT*>(ws + interval_bitmap_bytes(p.words, kPlain));
     PosT* sS = reinterpret_cast<PosT*>(ws + interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)));
     PosT* sE = sS + K;
-    // plain model: one byte per event and kind of mark (active starts, all starts) during pass 1, in the space of
-    // the difference array (2 (D + 1) <= (K + 2) sizeof(MemT) since D = K there)
+    // plain model: two bytes per event during pass 1 (active start, any start), in the space of the difference
+    // array when it is large enough (byte_marks)
     const uint32_t by_stride = ((uint32_t)p.D + 1u + 15u) & ~15u;
     uint8_t* by_act = reinterpret_cast<uint8_t*>(delta);
-    uint8_t* by_all = by_act + by_stride;
     constexpr uint32_t kFull = 0xFFFFFFFFu;
     const int nz = (int)(interval_clear_bytes(p.words, K, kPlain, sizeof(MemT)) >> 4);
 
@@ -161,7 +160,7 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
                         // are made from the bytes below; otherwise the marks go straight into them.
                         const uint32_t bit = 1u << (sv[i] & 31);
                         if (act) {
-                            if (kPlain && p.byte_marks) by_act[sv[i]] = 1;
+                            if (kPlain && p.byte_marks) by_act[2 * sv[i]] = 1;
                             else atomicOr(&bm_act[sv[i] >> 5], bit);
                             if (!kPlain && !((int64_t)sv[i] >= k && is_triangular_from((int64_t)sv[i] - k, k))) mask |= kIvStage;
                         }
@@ -170,7 +169,7 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
 #pragma unroll
                             for (int i2 = 0; i2 < i; ++i2) seen |= sv[i2] == sv[i];
                             if (!seen) {
-                                if (p.byte_marks) by_all[sv[i]] = 1;
+                                if (p.byte_marks) by_act[2 * sv[i] + 1] = 1;
                                 else atomicOr(&bm_all[sv[i] >> 5], bit);
                                 ++n_distinct;
                             }
@@ -191,15 +190,25 @@ __global__ void __launch_bounds__(32 * kIvMaxWarps) check_intervals_kernel(const
         }
         __syncwarp();
         if (kPlain && p.byte_marks) {
-            // bytes -> bitmaps: the warp reads 32 consecutive events, the ballot is their bitmap word; then the
-            // bytes, which borrowed the difference array, are cleared again
-            for (uint32_t wd = 0; wd < p.words; ++wd) {
-                const int32_t t = (int32_t)(wd * 32u) + lane;
-                const bool in = t <= p.D;
-                const uint32_t ba = __ballot_sync(kFull, in && by_act[t] != 0), bl = __ballot_sync(kFull, in && by_all[t] != 0);
-                if (lane == 0) {
-                    bm_act[wd] = ba;
-                    bm_all[wd] = bl;
+            // bytes -> bitmaps: the warp reads the byte pairs of 32 consecutive events, the two ballots are their
+            // bitmap words, kept by lane (word mod 32) and stored 32 words at a time; then the bytes, which
+            // borrowed the difference array, are cleared again
+            const uint16_t* by2 = reinterpret_cast<const uint16_t*>(by_act);
+            for (uint32_t w0 = 0; w0 < p.words; w0 += 32) {
+                uint32_t keep_a = 0, keep_l = 0;
+                const uint32_t w1 = min(p.words, w0 + 32u);
+                for (uint32_t wd = w0; wd < w1; ++wd) {
+                    const int32_t t = (int32_t)(wd * 32u) + lane;
+                    const uint32_t pr = t <= p.D ? (uint32_t)by2[t] : 0u;
+                    const uint32_t ba = __ballot_sync(kFull, (pr & 0xFFu) != 0), bl = __ballot_sync(kFull, (pr >> 8) != 0);
+                    if (lane == (int)(wd - w0)) {
+                        keep_a = ba;
+                        keep_l = bl;
+                    }
+                }
+                if (w0 + lane < w1) {
+                    bm_act[w0 + lane] = keep_a;
+                    bm_all[w0 + lane] = keep_l;
                 }
             }
             __syncwarp();
